@@ -1,0 +1,201 @@
+/*
+ * tts.h -- C-ABI of the B200 (sm_100a) verify-step library.
+ *
+ * The verify step of batched speculative decoding for test-time scaling: the target model
+ * scores N concurrent branches of one question (branch-wise parallelism, Section 3.2), each
+ * carrying gamma draft tokens plus one bonus position (sequence-wise parallelism, Section 3.2;
+ * "verify them in parallel while ensuring a lossless acceleration", Section 2).  The library
+ * covers the two parts of that step that are not weight GEMMs:
+ *   (1) GQA attention of the N*(gamma+1) query positions over a paged KV cache ("KV caches are
+ *       loaded from HBM", Section 3.1) whose prompt prefix is shared by all branches, and
+ *   (2) the speculative-sampling accept / residual-resample pass,
+ * plus the host-side answer aggregation (majority voting, Section 3.2; confidence-weighted
+ * variants, Section 4.6) and the greedy (B, gamma) search (Algorithm 1).
+ *
+ * Conventions
+ *   - Every function returns a tts_status (0 = OK, negative = error); no exceptions, no
+ *     process exit, no CPU fallback.
+ *   - "device" pointers are CUDA device memory on the context's device, owned by the caller,
+ *     16-byte aligned and densely packed in the stated layout.  The library never frees or
+ *     retains them.  "host" pointers are ordinary process memory.
+ *   - Device work is asynchronous on the context's stream; outputs are valid once the caller
+ *     has synchronised that stream.
+ *   - bf16 = 16-bit brain float, fp32 = IEEE binary32, i32 = int32_t.
+ */
+#ifndef TTS_H_
+#define TTS_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define TTS_API __attribute__((visibility("default")))
+#else
+#define TTS_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TTS_OK = 0,
+    TTS_ERR_INVALID = -1,        /* null pointer, size out of range, misaligned, prefix_len % page != 0 */
+    TTS_ERR_UNSUPPORTED = -2,    /* head_dim != 128, page_size != 16, unknown mask_kind / option */
+    TTS_ERR_CUDA = -3,           /* a CUDA call failed; tts_last_cuda_error() has the code */
+    TTS_ERR_DEVICE_BOUNDS = -4,  /* (via tts_last_status) a kernel saw a page id / token out of range */
+    TTS_ERR_DEVICE_TIMEOUT = -5  /* (via tts_last_status) a bounded device-side wait ran out */
+} tts_status;
+
+enum { TTS_MASK_CAUSAL = 0, TTS_MASK_TREE = 1 };
+enum { TTS_OUT_BF16 = 0, TTS_OUT_FP32 = 1 };
+/* Which attention kernel runs: AUTO picks tensor cores (tcgen05, TMEM accumulators) when the
+ * stacked query rows per KV head make it worthwhile and CUDA cores otherwise. */
+enum { TTS_ATTN_AUTO = 0, TTS_ATTN_SIMT = 1, TTS_ATTN_TCGEN05 = 2 };
+
+typedef struct tts_ctx tts_ctx;
+
+typedef struct {
+    int32_t n_q_heads;             /* Hq */
+    int32_t n_kv_heads;            /* Hkv, divides Hq; query head h reads KV head h / (Hq/Hkv) */
+    int32_t head_dim;              /* must be 128 */
+    int32_t page_size;             /* must be 16 tokens */
+    int32_t max_branches;          /* upper bound for n_branches (sizes the workspace) */
+    int32_t max_rows_per_branch;   /* upper bound for gamma+1 (or tree nodes) */
+    int32_t max_blocks_per_branch; /* row stride of block_table, in entries */
+    int32_t num_pages;             /* pages in each K / V pool; page ids must be < num_pages */
+    int32_t out_dtype;             /* TTS_OUT_BF16 (round to nearest even) or TTS_OUT_FP32 */
+    int32_t attn_impl;             /* TTS_ATTN_* */
+    float   softmax_scale;         /* 0 => 1/sqrt(head_dim) */
+    int32_t debug_bounds;          /* != 0: kernels range-check page ids and lengths, report through
+                                      tts_last_status instead of reading out of range */
+} tts_config;
+
+/* Creates a context on the CURRENT CUDA device and allocates its workspace there (split-KV
+ * partial results; a few MB to tens of MB depending on max_branches).  Host pointer out. */
+TTS_API int tts_create(const tts_config* cfg, tts_ctx** out);
+/* Frees the workspace.  The caller must have synchronised the stream first. */
+TTS_API int tts_destroy(tts_ctx* ctx);
+/* cuda_stream is a cudaStream_t passed as void*; NULL = the legacy default stream. */
+TTS_API int tts_set_stream(tts_ctx* ctx, void* cuda_stream);
+
+/*
+ * Verify-step attention for one layer (Section 3.1: the KV cache is streamed from HBM; Section
+ * 3.2: N branches x (gamma+1) positions are scored in one pass).  Exact softmax attention:
+ *   out[b][i][h] = sum_t softmax_t(scale * <q[b][i][h], K[t][h/G]>) * V[t][h/G]
+ * over the keys row i of branch b may see: all prefix tokens, and the private tokens
+ * j <= L_b - (gamma+1) + i of that branch (TTS_MASK_CAUSAL, bottom-right aligned).
+ *
+ *   q, out       device  [n_branches][gamma+1][Hq][128]  bf16 (out: cfg.out_dtype)
+ *   k_pages,     device  [num_pages][Hkv][16][128] bf16; slots no query may see (tail of a
+ *   v_pages              branch's last page, unused pages) may hold anything, NaN included
+ *   block_table  device  [n_branches][max_blocks_per_branch] i32: physical page of logical page
+ *                        j of branch b, logical order = prefix pages then private pages.  The
+ *                        first prefix_len/16 entries of every row must be equal (that equality
+ *                        is the sharing); entries past a branch's last page are ignored.
+ *   prefix_len   host    shared-prefix tokens, multiple of 16 (a ragged prompt tail belongs to
+ *                        the private part); may be 0
+ *   branch_lens  device  [n_branches] i32: private KV tokens of each branch INCLUDING the
+ *                        gamma+1 in-flight positions, whose K/V are already in the pages;
+ *                        precondition branch_lens[b] >= gamma+1
+ *   mask_kind    TTS_MASK_CAUSAL (TTS_MASK_TREE: use tts_verify_attn_tree)
+ * Errors: INVALID / UNSUPPORTED from host-side checks, CUDA on launch failure.  Device-side
+ * preconditions are checked only when cfg.debug_bounds != 0.
+ */
+TTS_API int tts_verify_attn(tts_ctx* ctx, const void* q, const void* k_pages, const void* v_pages,
+                    const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
+                    int n_branches, int gamma, int mask_kind, void* out);
+
+/*
+ * Tree verification (draft token trees, as produced by tree drafters such as the EAGLE-3 draft
+ * model used in Section 4.1): the last n_nodes private tokens of each branch are tree nodes;
+ * row i sees the prefix, the private tokens before the tree, itself and its ancestors.
+ *   tree_parents device [n_branches][n_nodes] i32, parent index in [-1, i); -1 = the node hangs
+ *                off the committed context.  q/out are [n_branches][n_nodes][Hq][128].
+ */
+TTS_API int tts_verify_attn_tree(tts_ctx* ctx, const void* q, const void* k_pages, const void* v_pages,
+                         const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
+                         const int32_t* tree_parents, int n_branches, int n_nodes, void* out);
+
+/*
+ * Speculative-sampling accept / resample (the lossless verification rule of the works cited in
+ * Section 2, "Speculative decoding").  Per branch b, with x_i = draft_tokens[b][i]:
+ *   accept x_i iff p_i(x_i) > 0 and u_i * q_i(x_i) <= p_i(x_i)  (one fp32 multiply), i = 0.. ;
+ *   accepted_len[b] = number accepted before the first rejection (0..gamma);
+ *   next_token[b]  = inverse-CDF draw with u_gamma from norm(max(0, p_k - q_k)) after a rejection
+ *                    at k (from p_k if that residual is identically 0), or from p_gamma (bonus
+ *                    token) when all gamma were accepted: the smallest x whose running sum of
+ *                    weights (fp64) exceeds u_gamma * total.
+ *   p_target device [n_branches][gamma+1][vocab] fp32     q_draft device [n_branches][gamma][vocab] fp32
+ *   draft_tokens device [n_branches][gamma] i32           uniforms device [n_branches][gamma+1] fp32 in [0,1)
+ *   accepted_len, next_token device [n_branches] i32.     vocab % 4 == 0; gamma may be 0.
+ */
+TTS_API int tts_accept(tts_ctx* ctx, const float* p_target, const float* q_draft,
+               const int32_t* draft_tokens, const float* uniforms, int n_branches, int gamma,
+               int vocab, int32_t* accepted_len, int32_t* next_token);
+
+/*
+ * Answer aggregation over the n branches of one question.  Host pointers, no GPU work.
+ *   tts_majority_vote: winner = most frequent answer (weights == NULL, Section 3.2) or the answer
+ *     with the largest weight sum ("vote" aggregation of Section 4.6); ties go to the answer whose
+ *     first occurrence has the lowest branch index.  votes = branches that gave the winner.
+ *   tts_confidence_max: answer of the single branch with the largest weight ("max" aggregation of
+ *     Section 4.6; ties: lowest branch index).
+ */
+TTS_API int tts_majority_vote(const int64_t* answers, const float* weights, int n, int64_t* winner,
+                      int* votes);
+TTS_API int tts_confidence_max(const int64_t* answers, const float* weights, int n, int64_t* winner,
+                       int* votes);
+
+/*
+ * Greedy search for the latency-optimal (B, gamma) (Algorithm 1).  Host only.  tts_task is called
+ * as tts_task(B, gamma, user) and returns the accuracy reached within the caller's latency budget;
+ * a negative return marks the point as unavailable (outside the caller's range).  Starts at
+ * (1, 0); each step evaluates (2B, gamma) and (B, gamma+1), moves to the better one (branch-wise
+ * on ties) if it improves, stops otherwise.  steps = loop iterations.
+ */
+typedef double (*tts_task_fn)(int n_branches, int gamma, void* user);
+TTS_API int tts_greedy_search(tts_task_fn tts_task, void* user, int* best_branches, int* best_gamma,
+                      double* best_acc, int* steps);
+
+/* Synchronises the stream and reads the device status word: TTS_OK, TTS_ERR_DEVICE_BOUNDS or
+ * TTS_ERR_DEVICE_TIMEOUT, written to *device_status; clears it.  Host pointers. */
+TTS_API int tts_last_status(tts_ctx* ctx, int* device_status);
+/* cudaError_t of the last failed CUDA call seen by this context (0 if none). */
+TTS_API int tts_last_cuda_error(tts_ctx* ctx);
+/* Number of kernels this context has launched since creation (host counter). */
+TTS_API int64_t tts_launch_count(tts_ctx* ctx);
+/*
+ * Profiling aid.  While enabled, every attention call records CUDA events on the context's stream
+ * before its main kernel, between the main kernel and the merge kernel, and after the merge (at
+ * most 4096 calls are kept).  tts_profile_read synchronises the stream, writes the mean duration
+ * in microseconds of the main kernel and of the merge kernel over the recorded calls and their
+ * number (host pointers), and forgets them.
+ */
+TTS_API int tts_profile_enable(tts_ctx* ctx, int on);
+TTS_API int tts_profile_read(tts_ctx* ctx, float* attn_main_us, float* attn_merge_us, int* n_calls);
+/* Static, NUL-terminated description of a tts_status. */
+TTS_API const char* tts_strerror(int status);
+
+/*
+ * One whole verify step from HOST buffers (the end-to-end path): for each of n_layers layers,
+ * copies that layer's q from pinned host memory, runs tts_verify_attn against that layer's
+ * device-resident K/V pools (the KV cache is state that lives in HBM, like the weights) and
+ * copies out back; then copies the probabilities, tokens and uniforms, runs tts_accept and
+ * copies the two result arrays back.  Synchronises before returning.
+ *   q_host, out_host   host  [n_layers][n_branches][gamma+1][Hq][128] bf16
+ *   k_pools, v_pools   host arrays of n_layers DEVICE pointers
+ *   block_table_host, branch_lens_host, p_target_host, q_draft_host, draft_tokens_host,
+ *   uniforms_host, accepted_len_host, next_token_host: host copies in the device layouts above.
+ * Staging buffers on the device are allocated inside the context on first use.
+ */
+TTS_API int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const void* const* k_pools,
+                         const void* const* v_pools, const int32_t* block_table_host,
+                         int prefix_len, const int32_t* branch_lens_host, int n_branches, int gamma,
+                         const float* p_target_host, const float* q_draft_host,
+                         const int32_t* draft_tokens_host, const float* uniforms_host, int vocab,
+                         void* out_host, int32_t* accepted_len_host, int32_t* next_token_host);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TTS_H_ */

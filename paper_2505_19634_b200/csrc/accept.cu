@@ -1,0 +1,194 @@
+// Speculative-sampling accept / resample: one CTA per branch.
+//
+//  1. warp 0 gathers p_i(x_i), q_i(x_i) for the gamma draft tokens and applies the test
+//     u_i * q <= p (single fp32 multiply) lane-parallel; a ballot gives the first rejection k.
+//  2. all warps sweep the one row pair that matters -- max(0, p_k - q_k) after a rejection, or
+//     p_gamma for the bonus token -- with 16-byte loads, 128 tokens per warp step, and leave one
+//     fp64 sum per 128-token tile in shared memory.  This is the only pass over HBM.
+//  3. warp 0 scans the tile sums (fp64), finds the tile where the running sum first exceeds
+//     u_gamma * Z, re-reads those 128 weights and finishes the inverse CDF inside the tile.
+#include "tts_internal.cuh"
+
+namespace tts {
+
+namespace {
+
+constexpr int kAccThreads = 1024;
+constexpr int kTileElems = 128;            // one warp step: 32 lanes x float4
+constexpr int kMaxTiles = 4096;            // vocab <= 524288
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ double warp_incl_scan(double v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        double n = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += n;
+    }
+    return v;
+}
+
+// residual weight of one token; mode_residual: max(0, p - q) in fp32, else p
+__device__ __forceinline__ float weight(float p, float q, bool residual) {
+    if (!residual) return p;
+    const float d = __fsub_rn(p, q);
+    return d > 0.f ? d : 0.f;
+}
+
+__global__ void __launch_bounds__(kAccThreads)
+accept_kernel(const float* __restrict__ p_target, const float* __restrict__ q_draft,
+              const int32_t* __restrict__ draft_tokens, const float* __restrict__ uniforms, int gamma,
+              int vocab, int32_t* __restrict__ accepted_len, int32_t* __restrict__ next_token,
+              int32_t* status) {
+    __shared__ double tile_sum[kMaxTiles];
+    __shared__ int s_k, s_last_pos, s_redo;
+
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float* P = p_target + (size_t)b * (gamma + 1) * vocab;
+    const float* Q = q_draft + (size_t)b * gamma * vocab;
+    const float* U = uniforms + (size_t)b * (gamma + 1);
+
+    // ---- 1. accept tests ----
+    if (warp == 0) {
+        int k = gamma;
+        for (int base = 0; base < gamma && k == gamma; base += 32) {
+            const int i = base + lane;
+            bool reject = false;
+            if (i < gamma) {
+                int x = draft_tokens[(size_t)b * gamma + i];
+                if (x < 0 || x >= vocab) { atomicMin(status, (int)TTS_ERR_DEVICE_BOUNDS); x = 0; }
+                const float p = P[(size_t)i * vocab + x];
+                const float q = Q[(size_t)i * vocab + x];
+                const float uq = __fmul_rn(U[i], q);
+                reject = !(p > 0.f && uq <= p);
+            }
+            const unsigned ballot = __ballot_sync(0xffffffffu, reject);
+            if (ballot) k = base + __ffs(ballot) - 1;
+        }
+        if (lane == 0) { s_k = k; s_last_pos = -1; s_redo = 0; accepted_len[b] = k; }
+    }
+    __syncthreads();
+    const int k = s_k;
+    const float* pk = P + (size_t)k * vocab;
+    const float* qk = Q + (size_t)(k < gamma ? k : 0) * vocab;
+    bool residual = k < gamma;
+    const int n_tiles = (vocab + kTileElems - 1) / kTileElems;
+
+    double Z = 0.0;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        // ---- 2. one sweep: per-tile fp64 sums ----
+        int last_pos = -1;
+        for (int j = warp; j < n_tiles; j += kAccThreads / 32) {
+            const int x0 = j * kTileElems + lane * 4;
+            double s = 0.0;
+            if (x0 < vocab) {                                   // vocab % 4 == 0: whole float4 in range
+                const float4 pv = __ldg(reinterpret_cast<const float4*>(pk + x0));
+                float4 qv = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (residual) qv = __ldg(reinterpret_cast<const float4*>(qk + x0));
+                const float w0 = weight(pv.x, qv.x, residual), w1 = weight(pv.y, qv.y, residual);
+                const float w2 = weight(pv.z, qv.z, residual), w3 = weight(pv.w, qv.w, residual);
+                s = (double)w0 + (double)w1 + (double)w2 + (double)w3;
+                if (w3 > 0.f) last_pos = x0 + 3; else if (w2 > 0.f) last_pos = x0 + 2;
+                else if (w1 > 0.f) last_pos = x0 + 1; else if (w0 > 0.f) last_pos = x0;
+            }
+            s = warp_sum(s);
+            if (lane == 0) tile_sum[j] = s;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xffffffffu, last_pos, o));
+        if (lane == 0 && last_pos >= 0) atomicMax(&s_last_pos, last_pos);
+        __syncthreads();
+
+        // ---- 3a. warp 0: total mass ----
+        if (warp == 0) {
+            const int per = (n_tiles + 31) / 32;
+            double c = 0.0;
+            for (int j = lane * per; j < min(n_tiles, (lane + 1) * per); ++j) c += tile_sum[j];
+            Z = warp_sum(c);
+            if (lane == 0) s_redo = (residual && !(Z > 0.0)) ? 1 : 0;
+        }
+        __syncthreads();
+        if (!s_redo) break;
+        residual = false;                                        // residual identically 0: draw from p_k
+        __syncthreads();
+        if (tid == 0) s_last_pos = -1;
+        __syncthreads();
+    }
+
+    // ---- 3b. warp 0: locate the crossing tile, then the token inside it ----
+    if (warp == 0) {
+        const double t = (double)U[gamma] * Z;
+        const int per = (n_tiles + 31) / 32;
+        const int j0 = lane * per, j1 = min(n_tiles, (lane + 1) * per);
+        double c = 0.0;
+        for (int j = j0; j < j1; ++j) c += tile_sum[j];
+        const double incl = warp_incl_scan(c, lane);
+        const unsigned hit = __ballot_sync(0xffffffffu, incl > t);
+        int chosen = -1;
+        if (hit) {
+            const int src = __ffs(hit) - 1;
+            int tile = -1;
+            double base = 0.0;
+            if (lane == src) {
+                double run = incl - c;
+                for (int j = j0; j < j1; ++j) {
+                    const double nxt = run + tile_sum[j];
+                    if (nxt > t) { tile = j; base = run; break; }
+                    run = nxt;
+                }
+            }
+            tile = __shfl_sync(0xffffffffu, tile, src);
+            base = __shfl_sync(0xffffffffu, base, src);
+            if (tile >= 0) {
+                const int x0 = tile * kTileElems + lane * 4;
+                float w[4] = {0.f, 0.f, 0.f, 0.f};
+                if (x0 < vocab) {
+                    const float4 pv = *reinterpret_cast<const float4*>(pk + x0);
+                    float4 qv = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (residual) qv = *reinterpret_cast<const float4*>(qk + x0);
+                    w[0] = weight(pv.x, qv.x, residual); w[1] = weight(pv.y, qv.y, residual);
+                    w[2] = weight(pv.z, qv.z, residual); w[3] = weight(pv.w, qv.w, residual);
+                }
+                const double ls = (double)w[0] + (double)w[1] + (double)w[2] + (double)w[3];
+                const double lincl = warp_incl_scan(ls, lane);
+                const unsigned lhit = __ballot_sync(0xffffffffu, base + lincl > t);
+                if (lhit) {
+                    const int ls_src = __ffs(lhit) - 1;
+                    int x = -1;
+                    if (lane == ls_src) {
+                        double run = base + (lincl - ls);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            run += (double)w[e];
+                            if (x < 0 && run > t) x = x0 + e;
+                        }
+                        if (x < 0)                       // summation order left no crossing here
+                            x = w[3] > 0.f ? x0 + 3 : (w[2] > 0.f ? x0 + 2 : (w[1] > 0.f ? x0 + 1 : x0));
+                    }
+                    chosen = __shfl_sync(0xffffffffu, x, ls_src);
+                }
+            }
+        }
+        if (lane == 0) {
+            if (chosen < 0) chosen = s_last_pos >= 0 ? s_last_pos : vocab - 1;   // rounding left no crossing
+            next_token[b] = chosen;
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_accept(const float* p_target, const float* q_draft, const int32_t* draft_tokens,
+                          const float* uniforms, int n_branches, int gamma, int vocab,
+                          int32_t* accepted_len, int32_t* next_token, int32_t* status,
+                          cudaStream_t st) {
+    accept_kernel<<<n_branches, kAccThreads, 0, st>>>(p_target, q_draft, draft_tokens, uniforms,
+                                                      gamma, vocab, accepted_len, next_token, status);
+    return cudaGetLastError();
+}
+
+}  // namespace tts

@@ -1,0 +1,96 @@
+// Merge of the split-KV partial results: for every output row, the log-sum-exp combination of
+// the pieces of its prefix segment and of its private segment, normalisation and the cast to
+// the output type.  One warp per output row, four head dims per lane.
+#include "tts_internal.cuh"
+
+namespace tts {
+
+namespace {
+
+constexpr int kRowsPerBlock = 4;
+
+__global__ void __launch_bounds__(kRowsPerBlock * 32) attn_combine_kernel(const AttnParams p) {
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * kRowsPerBlock + (threadIdx.x >> 5);     // (b, i, h) flattened
+    if (row >= p.N * p.R * p.Hq) return;
+    const int h = row % p.Hq, i = (row / p.Hq) % p.R, b = row / (p.Hq * p.R);
+    const int kvh = h / p.G, gq = h % p.G;
+
+    // tiles of the branches before b, of b, and of all branches (lanes stride over branches)
+    int before = 0, all = 0;
+    for (int bb = lane; bb < p.N; bb += 32) {
+        int L = p.branch_lens[bb];
+        const int t = ceil_div(L < 0 ? 0 : L, p.tile_tokens);
+        all += t;
+        if (bb < b) before += t;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        before += __shfl_xor_sync(0xffffffffu, before, o);
+        all += __shfl_xor_sync(0xffffffffu, all, o);
+    }
+    const int tiles_b = ceil_div(max(p.branch_lens[b], 0), p.tile_tokens);
+    const int per = p.Hkv * p.n_rb_priv;
+    const int pre_total = p.n_pre * p.tiles_pre;
+    const int total = pre_total + per * all;
+    const int tpc = ceil_div(total, p.grid);
+
+    float m_run = -INFINITY, l_run = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+
+    auto merge = [&](const float* o_base, const float2* ml_base, int stride, int seg_local, int r,
+                     int t_begin, int n_tiles) {
+        if (n_tiles <= 0) return;
+        const int c0 = t_begin / tpc, c1 = (t_begin + n_tiles - 1) / tpc;
+        for (int c = c0; c <= c1; ++c) {
+            const size_t id = (size_t)seg_local + c;
+            const float2 ml = ml_base[id * stride + r];
+            if (!(ml.y > 0.f)) continue;                  // piece saw no visible key for this row
+            const float4 o = *reinterpret_cast<const float4*>(
+                o_base + (id * stride + r) * kHeadDim + lane * 4);
+            const float m_new = fmaxf(m_run, ml.x);
+            const float a = (m_run == -INFINITY) ? 0.f : exp2f(m_run - m_new);
+            const float w = exp2f(ml.x - m_new);
+            acc.x = acc.x * a + o.x * w; acc.y = acc.y * a + o.y * w;
+            acc.z = acc.z * a + o.z * w; acc.w = acc.w * a + o.w * w;
+            l_run = l_run * a + ml.y * w;
+            m_run = m_new;
+        }
+    };
+
+    const int r_priv = i * p.G + gq;
+    if (p.n_pre > 0) {
+        const int pr = b * p.nr + r_priv;
+        const int rb = pr / p.rb_rows, r = pr % p.rb_rows;
+        const int seg = kvh * p.n_rb_pre + rb;
+        merge(p.part_o_pre, p.part_ml_pre, p.pre_stride, seg, r, seg * p.tiles_pre, p.tiles_pre);
+    }
+    {
+        const int rb = r_priv / p.rb_rows, r = r_priv % p.rb_rows;
+        const int within = kvh * p.n_rb_priv + rb;
+        const int seg = b * per + within;
+        merge(p.part_o_priv, p.part_ml_priv, p.priv_stride, seg, r, pre_total + per * before + within * tiles_b, tiles_b);
+    }
+
+    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+    acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+    if (p.out_dtype == TTS_OUT_FP32) {
+        *reinterpret_cast<float4*>(static_cast<float*>(p.out) + (size_t)row * kHeadDim + lane * 4) = acc;
+    } else {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+        uint2 pk;
+        pk.x = *reinterpret_cast<unsigned*>(&lo);
+        pk.y = *reinterpret_cast<unsigned*>(&hi);
+        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.out) + (size_t)row * kHeadDim + lane * 4) = pk;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_attn_combine(const AttnParams& p, cudaStream_t st) {
+    const int rows = p.N * p.R * p.Hq;
+    attn_combine_kernel<<<ceil_div(rows, kRowsPerBlock), kRowsPerBlock * 32, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace tts

@@ -1,0 +1,441 @@
+// C-ABI layer: argument checks, context and workspace management, kernel launches, and the
+// host-only helpers (answer aggregation, greedy search).  See include/tts.h for the contract.
+#include <math.h>
+#include <new>
+#include <stdlib.h>
+#include <string.h>
+
+#include "tts_internal.cuh"
+
+using namespace tts;
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int cuda_fail(Ctx* c, cudaError_t e) {
+    if (c) c->last_cuda_error = (int)e;
+    return TTS_ERR_CUDA;
+}
+
+// Row-block size and tile length the chosen kernel works with.
+struct Plan { int impl, rb_rows, tile_tokens, grid; };
+
+Plan make_plan(const Ctx* c, int nr) {
+    Plan pl;
+    int impl = c->cfg.attn_impl;
+    if (impl == TTS_ATTN_AUTO) impl = umma_available() && nr >= kUmmaMinRows ? TTS_ATTN_TCGEN05 : TTS_ATTN_SIMT;
+    pl.impl = impl;
+    if (impl == TTS_ATTN_TCGEN05) {
+        pl.rb_rows = kUmmaRows; pl.tile_tokens = kUmmaTileTokens; pl.grid = c->n_sms;
+    } else {
+        pl.rb_rows = simt_rb_rows(nr); pl.tile_tokens = kSimtTileTokens; pl.grid = c->n_sms * 3;
+    }
+    return pl;
+}
+
+void free_workspace(Ctx* c) {
+    cudaFree(c->part_o_pre); cudaFree(c->part_ml_pre); cudaFree(c->part_o_priv); cudaFree(c->part_ml_priv);
+    c->part_o_pre = c->part_o_priv = nullptr; c->part_ml_pre = c->part_ml_priv = nullptr;
+    c->pre_rows = c->priv_rows = 0;
+}
+
+// Partial-result rows one call needs: every piece reserves min(rb_rows, rows of its segment kind).
+void workspace_rows(int N, int Hkv, int nr, int rb_rows, int grid, size_t* pre, size_t* priv) {
+    const long n_rb_pre = ((long)N * nr + rb_rows - 1) / rb_rows;
+    const long n_rb_priv = (nr + rb_rows - 1) / rb_rows;
+    const long pre_stride = (long)N * nr < rb_rows ? (long)N * nr : rb_rows;
+    const long priv_stride = nr < rb_rows ? nr : rb_rows;
+    *pre = (size_t)(Hkv * n_rb_pre + grid) * pre_stride;
+    *priv = (size_t)((long)N * Hkv * n_rb_priv + grid) * priv_stride;
+}
+
+// Workspace for the largest problem the config allows, whichever kernel a call ends up using.
+cudaError_t alloc_workspace(Ctx* c) {
+    const tts_config& f = c->cfg;
+    const int G = f.n_q_heads / f.n_kv_heads;
+    const int nr = f.max_rows_per_branch * G;
+    size_t pre = 0, priv = 0;
+    const int cand_rb[4] = {8, 16, 32, kUmmaRows};
+    for (int k = 0; k < 4; ++k) {
+        size_t a, b;
+        workspace_rows(f.max_branches, f.n_kv_heads, nr, cand_rb[k], c->n_sms * 3, &a, &b);
+        pre = a > pre ? a : pre; priv = b > priv ? b : priv;
+    }
+    cudaError_t e;
+    if ((e = cudaMalloc(&c->part_o_pre, pre * kHeadDim * sizeof(float))) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&c->part_ml_pre, pre * sizeof(float2))) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&c->part_o_priv, priv * kHeadDim * sizeof(float))) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&c->part_ml_priv, priv * sizeof(float2))) != cudaSuccess) return e;
+    c->pre_rows = pre; c->priv_rows = priv;
+    return cudaSuccess;
+}
+
+int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
+                const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
+                const int32_t* tree_parents, int n_branches, int rows, void* out) {
+    if (!c || !q || !k_pages || !v_pages || !block_table || !branch_lens || !out) return TTS_ERR_INVALID;
+    const tts_config& f = c->cfg;
+    if (n_branches < 1 || n_branches > f.max_branches) return TTS_ERR_INVALID;
+    if (rows < 1 || rows > f.max_rows_per_branch) return TTS_ERR_INVALID;
+    if (tree_parents && rows > kMaxTreeRows) return TTS_ERR_UNSUPPORTED;
+    if (!tree_parents && rows > kMaxTreeRows) return TTS_ERR_UNSUPPORTED;
+    if (prefix_len < 0 || prefix_len % f.page_size != 0) return TTS_ERR_INVALID;
+    if (prefix_len / f.page_size > f.max_blocks_per_branch) return TTS_ERR_INVALID;
+    if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(out) ||
+        (reinterpret_cast<uintptr_t>(block_table) & 3u) || (reinterpret_cast<uintptr_t>(branch_lens) & 3u))
+        return TTS_ERR_INVALID;
+
+    const int G = f.n_q_heads / f.n_kv_heads;
+    const int nr = rows * G;
+    const Plan pl = make_plan(c, nr);
+
+    {
+        size_t need_pre, need_priv;
+        workspace_rows(n_branches, f.n_kv_heads, nr, pl.rb_rows, pl.grid, &need_pre, &need_priv);
+        if (need_pre > c->pre_rows || need_priv > c->priv_rows) return TTS_ERR_INVALID;
+    }
+    cudaError_t e;
+
+    AttnParams p;
+    memset(&p, 0, sizeof p);
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k_pages = static_cast<const __nv_bfloat16*>(k_pages);
+    p.v_pages = static_cast<const __nv_bfloat16*>(v_pages);
+    p.block_table = block_table; p.branch_lens = branch_lens; p.tree_parents = tree_parents;
+    p.out = out;
+    p.part_o_pre = c->part_o_pre; p.part_ml_pre = c->part_ml_pre;
+    p.part_o_priv = c->part_o_priv; p.part_ml_priv = c->part_ml_priv;
+    p.status = c->d_status;
+    p.N = n_branches; p.R = rows; p.Hq = f.n_q_heads; p.Hkv = f.n_kv_heads; p.G = G; p.nr = nr;
+    p.P = prefix_len; p.max_blocks = f.max_blocks_per_branch; p.num_pages = f.num_pages;
+    p.rb_rows = pl.rb_rows;
+    p.pre_stride = n_branches * nr < pl.rb_rows ? n_branches * nr : pl.rb_rows;
+    p.priv_stride = nr < pl.rb_rows ? nr : pl.rb_rows;
+    p.n_rb_pre = ceil_div(n_branches * nr, pl.rb_rows);
+    p.n_rb_priv = ceil_div(nr, pl.rb_rows);
+    p.n_pre = prefix_len > 0 ? f.n_kv_heads * p.n_rb_pre : 0;
+    p.tile_tokens = pl.tile_tokens;
+    p.tiles_pre = ceil_div(prefix_len, pl.tile_tokens);
+    p.grid = pl.grid;
+    p.out_dtype = f.out_dtype; p.debug = f.debug_bounds;
+    const float scale = f.softmax_scale > 0.f ? f.softmax_scale : 1.0f / sqrtf((float)f.head_dim);
+    p.scale_log2 = scale * 1.4426950408889634f;
+
+    const bool prof = c->profiling && c->prof_ev && c->prof_n < kProfMaxCalls;
+    cudaEvent_t* ev = prof ? c->prof_ev + 3 * c->prof_n : nullptr;
+    if (prof) cudaEventRecord(ev[0], c->stream);
+    if (pl.impl == TTS_ATTN_TCGEN05) {
+        if (!umma_available()) return TTS_ERR_UNSUPPORTED;
+        e = launch_attn_umma(c, p, c->stream);
+    } else {
+        e = launch_attn_simt(p, c->stream);
+    }
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->launches += 1;
+    if (prof) cudaEventRecord(ev[1], c->stream);
+    e = launch_attn_combine(p, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->launches += 1;
+    if (prof) { cudaEventRecord(ev[2], c->stream); c->prof_n += 1; }
+    return TTS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int tts_create(const tts_config* cfg, tts_ctx** out) {
+    if (!cfg || !out) return TTS_ERR_INVALID;
+    *out = nullptr;
+    if (cfg->head_dim != kHeadDim || cfg->page_size != kPage) return TTS_ERR_UNSUPPORTED;
+    if (cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 || cfg->n_q_heads % cfg->n_kv_heads != 0) return TTS_ERR_INVALID;
+    if (cfg->max_branches < 1 || cfg->max_branches > kMaxBranches) return TTS_ERR_INVALID;
+    if (cfg->max_rows_per_branch < 1 || cfg->max_rows_per_branch > kMaxTreeRows) return TTS_ERR_INVALID;
+    if (cfg->max_blocks_per_branch < 1 || cfg->num_pages < 1) return TTS_ERR_INVALID;
+    if (cfg->out_dtype != TTS_OUT_BF16 && cfg->out_dtype != TTS_OUT_FP32) return TTS_ERR_UNSUPPORTED;
+    if (cfg->attn_impl < TTS_ATTN_AUTO || cfg->attn_impl > TTS_ATTN_TCGEN05) return TTS_ERR_UNSUPPORTED;
+    if (!(cfg->softmax_scale >= 0.f)) return TTS_ERR_INVALID;
+
+    Ctx* c = new (std::nothrow) Ctx();
+    if (!c) return TTS_ERR_INVALID;
+    memset(c, 0, sizeof *c);
+    c->cfg = *cfg;
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, c->device);
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_status, sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(int32_t));
+    if (e == cudaSuccess) e = alloc_workspace(c);
+    if (e != cudaSuccess) {
+        free_workspace(c);
+        cudaFree(c->d_status);
+        delete c;
+        return TTS_ERR_CUDA;
+    }
+    *out = reinterpret_cast<tts_ctx*>(c);
+    return TTS_OK;
+}
+
+int tts_destroy(tts_ctx* ctx) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c) return TTS_ERR_INVALID;
+    free_workspace(c);
+    cudaFree(c->d_status);
+    cudaFree(c->stage);
+    if (c->prof_ev) {
+        for (int i = 0; i < 3 * kProfMaxCalls; ++i) if (c->prof_ev[i]) cudaEventDestroy(c->prof_ev[i]);
+        free(c->prof_ev);
+    }
+    umma_release(c);
+    delete c;
+    return TTS_OK;
+}
+
+int tts_set_stream(tts_ctx* ctx, void* cuda_stream) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c) return TTS_ERR_INVALID;
+    c->stream = static_cast<cudaStream_t>(cuda_stream);
+    return TTS_OK;
+}
+
+int tts_verify_attn(tts_ctx* ctx, const void* q, const void* k_pages, const void* v_pages,
+                    const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
+                    int n_branches, int gamma, int mask_kind, void* out) {
+    if (mask_kind == TTS_MASK_TREE) return TTS_ERR_UNSUPPORTED;     // needs parents: tts_verify_attn_tree
+    if (mask_kind != TTS_MASK_CAUSAL) return TTS_ERR_UNSUPPORTED;
+    if (gamma < 0) return TTS_ERR_INVALID;
+    return attn_common(reinterpret_cast<Ctx*>(ctx), q, k_pages, v_pages, block_table, prefix_len,
+                       branch_lens, nullptr, n_branches, gamma + 1, out);
+}
+
+int tts_verify_attn_tree(tts_ctx* ctx, const void* q, const void* k_pages, const void* v_pages,
+                         const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
+                         const int32_t* tree_parents, int n_branches, int n_nodes, void* out) {
+    if (!tree_parents) return TTS_ERR_INVALID;
+    return attn_common(reinterpret_cast<Ctx*>(ctx), q, k_pages, v_pages, block_table, prefix_len,
+                       branch_lens, tree_parents, n_branches, n_nodes, out);
+}
+
+int tts_accept(tts_ctx* ctx, const float* p_target, const float* q_draft, const int32_t* draft_tokens,
+               const float* uniforms, int n_branches, int gamma, int vocab, int32_t* accepted_len,
+               int32_t* next_token) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !p_target || !uniforms || !accepted_len || !next_token) return TTS_ERR_INVALID;
+    if (gamma < 0 || n_branches < 1) return TTS_ERR_INVALID;
+    if (gamma > 0 && (!q_draft || !draft_tokens)) return TTS_ERR_INVALID;
+    if (vocab < 4 || vocab % 4 != 0 || vocab > 524288) return TTS_ERR_INVALID;
+    if (!aligned16(p_target) || (q_draft && !aligned16(q_draft))) return TTS_ERR_INVALID;
+    cudaError_t e = launch_accept(p_target, q_draft, draft_tokens, uniforms, n_branches, gamma, vocab,
+                                  accepted_len, next_token, c->d_status, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->launches += 1;
+    return TTS_OK;
+}
+
+static int vote_impl(const int64_t* answers, const float* weights, int n, int mode, int64_t* winner,
+                     int* votes) {
+    if (!answers || !winner || n < 1 || (mode == 1 && !weights)) return TTS_ERR_INVALID;
+    int best = -1;
+    double best_score = 0.0;
+    if (mode == 1) {
+        for (int i = 0; i < n; ++i)
+            if (best < 0 || (double)weights[i] > best_score) { best = i; best_score = weights[i]; }
+    } else {
+        // O(n^2) on purpose: n is the number of branches (<= a few hundred), no allocation
+        for (int i = 0; i < n; ++i) {
+            bool seen = false;
+            for (int j = 0; j < i && !seen; ++j) seen = answers[j] == answers[i];
+            if (seen) continue;
+            double s = 0.0;
+            for (int j = i; j < n; ++j)
+                if (answers[j] == answers[i]) s += weights ? (double)weights[j] : 1.0;
+            if (best < 0 || s > best_score) { best = i; best_score = s; }
+        }
+    }
+    int count = 0;
+    for (int j = 0; j < n; ++j) count += answers[j] == answers[best];
+    *winner = answers[best];
+    if (votes) *votes = count;
+    return TTS_OK;
+}
+
+int tts_majority_vote(const int64_t* answers, const float* weights, int n, int64_t* winner, int* votes) {
+    return vote_impl(answers, weights, n, 0, winner, votes);
+}
+
+int tts_confidence_max(const int64_t* answers, const float* weights, int n, int64_t* winner, int* votes) {
+    return vote_impl(answers, weights, n, 1, winner, votes);
+}
+
+int tts_greedy_search(tts_task_fn tts_task, void* user, int* best_branches, int* best_gamma,
+                      double* best_acc, int* steps) {
+    if (!tts_task || !best_branches || !best_gamma) return TTS_ERR_INVALID;
+    int B = 1, gamma = 0, n_steps = 0;
+    double acc = tts_task(B, gamma, user);
+    for (;;) {
+        ++n_steps;
+        const double acc_b = B <= (1 << 29) ? tts_task(2 * B, gamma, user) : -1.0;
+        const double acc_g = tts_task(B, gamma + 1, user);
+        int nb, ng; double nacc;
+        if (acc_b >= acc_g) { nb = 2 * B; ng = gamma; nacc = acc_b; }
+        else                { nb = B; ng = gamma + 1; nacc = acc_g; }
+        if (nacc > acc && nacc >= 0.0) { B = nb; gamma = ng; acc = nacc; }
+        else break;
+    }
+    *best_branches = B; *best_gamma = gamma;
+    if (best_acc) *best_acc = acc;
+    if (steps) *steps = n_steps;
+    return TTS_OK;
+}
+
+int tts_last_status(tts_ctx* ctx, int* device_status) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !device_status) return TTS_ERR_INVALID;
+    int32_t h = 0;
+    cudaError_t e = cudaMemcpyAsync(&h, c->d_status, sizeof h, cudaMemcpyDeviceToHost, c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->d_status, 0, sizeof h, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    *device_status = h;
+    return TTS_OK;
+}
+
+int tts_profile_enable(tts_ctx* ctx, int on) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c) return TTS_ERR_INVALID;
+    if (on && !c->prof_ev) {
+        c->prof_ev = static_cast<cudaEvent_t*>(calloc(3 * kProfMaxCalls, sizeof(cudaEvent_t)));
+        if (!c->prof_ev) return TTS_ERR_INVALID;
+        for (int i = 0; i < 3 * kProfMaxCalls; ++i) {
+            cudaError_t e = cudaEventCreate(&c->prof_ev[i]);
+            if (e != cudaSuccess) return cuda_fail(c, e);
+        }
+    }
+    c->profiling = on ? 1 : 0;
+    c->prof_n = 0;
+    return TTS_OK;
+}
+
+int tts_profile_read(tts_ctx* ctx, float* attn_main_us, float* attn_merge_us, int* n_calls) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !attn_main_us || !attn_merge_us || !n_calls) return TTS_ERR_INVALID;
+    cudaError_t e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    double a = 0.0, b = 0.0;
+    for (int i = 0; i < c->prof_n; ++i) {
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, c->prof_ev[3 * i], c->prof_ev[3 * i + 1]); a += ms;
+        cudaEventElapsedTime(&ms, c->prof_ev[3 * i + 1], c->prof_ev[3 * i + 2]); b += ms;
+    }
+    *n_calls = c->prof_n;
+    *attn_main_us = c->prof_n ? (float)(a * 1e3 / c->prof_n) : 0.f;
+    *attn_merge_us = c->prof_n ? (float)(b * 1e3 / c->prof_n) : 0.f;
+    c->prof_n = 0;
+    return TTS_OK;
+}
+
+int tts_last_cuda_error(tts_ctx* ctx) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    return c ? c->last_cuda_error : 0;
+}
+
+int64_t tts_launch_count(tts_ctx* ctx) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    return c ? c->launches : 0;
+}
+
+const char* tts_strerror(int status) {
+    switch (status) {
+        case TTS_OK: return "ok";
+        case TTS_ERR_INVALID: return "invalid argument";
+        case TTS_ERR_UNSUPPORTED: return "unsupported configuration";
+        case TTS_ERR_CUDA: return "CUDA call failed";
+        case TTS_ERR_DEVICE_BOUNDS: return "device-side bounds check failed";
+        case TTS_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const void* const* k_pools,
+                         const void* const* v_pools, const int32_t* block_table_host, int prefix_len,
+                         const int32_t* branch_lens_host, int n_branches, int gamma,
+                         const float* p_target_host, const float* q_draft_host,
+                         const int32_t* draft_tokens_host, const float* uniforms_host, int vocab,
+                         void* out_host, int32_t* accepted_len_host, int32_t* next_token_host) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || n_layers < 1 || !q_host || !k_pools || !v_pools || !block_table_host || !branch_lens_host ||
+        !p_target_host || !uniforms_host || !out_host || !accepted_len_host || !next_token_host)
+        return TTS_ERR_INVALID;
+    if (gamma < 0 || (gamma > 0 && (!q_draft_host || !draft_tokens_host))) return TTS_ERR_INVALID;
+    if (n_branches < 1 || n_branches > c->cfg.max_branches || gamma + 1 > c->cfg.max_rows_per_branch)
+        return TTS_ERR_INVALID;
+    if (vocab < 4 || vocab % 4 != 0) return TTS_ERR_INVALID;
+    const tts_config& f = c->cfg;
+    const size_t out_elt = f.out_dtype == TTS_OUT_FP32 ? 4 : 2;
+    const size_t q_layer = (size_t)n_branches * (gamma + 1) * f.n_q_heads * kHeadDim * 2;
+    const size_t o_layer = (size_t)n_branches * (gamma + 1) * f.n_q_heads * kHeadDim * out_elt;
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    const size_t bt_b = up((size_t)n_branches * f.max_blocks_per_branch * 4), bl_b = up((size_t)n_branches * 4);
+    const size_t pt_b = up((size_t)n_branches * (gamma + 1) * vocab * 4);
+    const size_t qd_b = up((size_t)n_branches * gamma * vocab * 4);
+    const size_t dt_b = up((size_t)n_branches * gamma * 4), un_b = up((size_t)n_branches * (gamma + 1) * 4);
+    const size_t res_b = up((size_t)n_branches * 4);
+    const size_t need = up(q_layer) * n_layers + up(o_layer) * n_layers + bt_b + bl_b + pt_b + qd_b + dt_b +
+                        un_b + 2 * res_b;
+    cudaError_t e;
+    if (c->stage_bytes < need) {
+        cudaFree(c->stage); c->stage = nullptr; c->stage_bytes = 0;
+        if ((e = cudaMalloc(&c->stage, need)) != cudaSuccess) return cuda_fail(c, e);
+        c->stage_bytes = need;
+    }
+    char* base = static_cast<char*>(c->stage);
+    char* d_q = base;               base += up(q_layer) * n_layers;
+    char* d_o = base;               base += up(o_layer) * n_layers;
+    int32_t* d_bt = (int32_t*)base; base += bt_b;
+    int32_t* d_bl = (int32_t*)base; base += bl_b;
+    float* d_pt = (float*)base;     base += pt_b;
+    float* d_qd = (float*)base;     base += qd_b;
+    int32_t* d_dt = (int32_t*)base; base += dt_b;
+    float* d_un = (float*)base;     base += un_b;
+    int32_t* d_al = (int32_t*)base; base += res_b;
+    int32_t* d_nt = (int32_t*)base;
+
+    cudaStream_t st = c->stream;
+#define TTS_CK(x) do { e = (x); if (e != cudaSuccess) return cuda_fail(c, e); } while (0)
+    TTS_CK(cudaMemcpyAsync(d_bt, block_table_host, (size_t)n_branches * f.max_blocks_per_branch * 4, cudaMemcpyHostToDevice, st));
+    TTS_CK(cudaMemcpyAsync(d_bl, branch_lens_host, (size_t)n_branches * 4, cudaMemcpyHostToDevice, st));
+    // all layers' queries in one copy (they are contiguous on the host)
+    if (up(q_layer) == q_layer) {
+        TTS_CK(cudaMemcpyAsync(d_q, q_host, q_layer * n_layers, cudaMemcpyHostToDevice, st));
+    } else {
+        for (int l = 0; l < n_layers; ++l)
+            TTS_CK(cudaMemcpyAsync(d_q + up(q_layer) * l, (const char*)q_host + q_layer * l, q_layer, cudaMemcpyHostToDevice, st));
+    }
+    for (int l = 0; l < n_layers; ++l) {
+        int rc = tts_verify_attn(ctx, d_q + up(q_layer) * l, k_pools[l], v_pools[l], d_bt, prefix_len, d_bl,
+                                 n_branches, gamma, TTS_MASK_CAUSAL, d_o + up(o_layer) * l);
+        if (rc != TTS_OK) return rc;
+    }
+    if (up(o_layer) == o_layer) {
+        TTS_CK(cudaMemcpyAsync(out_host, d_o, o_layer * n_layers, cudaMemcpyDeviceToHost, st));
+    } else {
+        for (int l = 0; l < n_layers; ++l)
+            TTS_CK(cudaMemcpyAsync((char*)out_host + o_layer * l, d_o + up(o_layer) * l, o_layer, cudaMemcpyDeviceToHost, st));
+    }
+    TTS_CK(cudaMemcpyAsync(d_pt, p_target_host, (size_t)n_branches * (gamma + 1) * vocab * 4, cudaMemcpyHostToDevice, st));
+    if (gamma > 0) {
+        TTS_CK(cudaMemcpyAsync(d_qd, q_draft_host, (size_t)n_branches * gamma * vocab * 4, cudaMemcpyHostToDevice, st));
+        TTS_CK(cudaMemcpyAsync(d_dt, draft_tokens_host, (size_t)n_branches * gamma * 4, cudaMemcpyHostToDevice, st));
+    }
+    TTS_CK(cudaMemcpyAsync(d_un, uniforms_host, (size_t)n_branches * (gamma + 1) * 4, cudaMemcpyHostToDevice, st));
+    int rc = tts_accept(ctx, d_pt, gamma > 0 ? d_qd : nullptr, gamma > 0 ? d_dt : nullptr, d_un, n_branches, gamma,
+                        vocab, d_al, d_nt);
+    if (rc != TTS_OK) return rc;
+    TTS_CK(cudaMemcpyAsync(accepted_len_host, d_al, (size_t)n_branches * 4, cudaMemcpyDeviceToHost, st));
+    TTS_CK(cudaMemcpyAsync(next_token_host, d_nt, (size_t)n_branches * 4, cudaMemcpyDeviceToHost, st));
+    TTS_CK(cudaStreamSynchronize(st));
+#undef TTS_CK
+    return TTS_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,193 @@
+// Internal declarations shared by the kernels and the C-ABI layer (not installed).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tts.h"
+
+namespace tts {
+
+constexpr int kHeadDim = 128;
+constexpr int kPage = 16;
+constexpr int kMaxTreeRows = 64;      // rows per branch that may carry an explicit visibility mask
+constexpr int kMaxBranches = 1024;
+
+// Work decomposition of one attention call.
+//
+// A *segment* is (KV head, block of <= rb_rows stacked query rows, run of KV tokens):
+//   prefix segments   s = kvh * n_rb_pre + rb            rows = all branches' rows, stacked
+//                                                          (b, i, g) -> b*nr + i*G + g; every row
+//                                                          sees every prefix token (no mask)
+//   private segments  s = n_pre + (b*Hkv + kvh) * n_rb_priv + rb   rows = (i, g) -> i*G + g
+// Each segment is cut into tiles of tile_tokens KV tokens; all tiles of all segments form one
+// global list, and CTA c of a persistent grid owns the contiguous run [c*tpc, (c+1)*tpc) of it
+// (tpc = ceil(total / grid)).  The run of one CTA inside one segment is a *piece*; it produces
+// one partial result (running max m, sum l, unnormalised O) per row.  Because segments and CTAs
+// advance together along the list, (segment + CTA) is a unique index for every piece, so no
+// scan over pieces is needed to place them in the workspace.
+struct AttnParams {
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* k_pages;
+    const __nv_bfloat16* v_pages;
+    const int32_t* block_table;
+    const int32_t* branch_lens;
+    const int32_t* tree_parents;   // null for causal
+    void* out;
+    float* part_o_pre;    // [n_pre + grid][pre_stride][128]
+    float2* part_ml_pre;  // [n_pre + grid][pre_stride]      (m in log2 units, l)
+    float* part_o_priv;   // [N*Hkv*n_rb_priv + grid][priv_stride][128]
+    float2* part_ml_priv;
+    int32_t* status;      // device status word
+    int N, R, Hq, Hkv, G, nr;      // nr = R*G rows per (branch, kv head)
+    int P;                          // prefix tokens
+    int max_blocks, num_pages;
+    int rb_rows;                    // rows per row block
+    int pre_stride, priv_stride;    // rows reserved per piece: min(rb_rows, N*nr) / min(rb_rows, nr)
+    int n_rb_pre, n_rb_priv;        // row blocks per prefix kv head / per (branch, kv head)
+    int n_pre;                      // prefix segments (0 when P == 0)
+    int tiles_pre;                  // tiles per prefix segment
+    int tile_tokens;
+    int grid;                       // CTAs of the main kernel
+    int out_dtype, debug;
+    float scale_log2;               // softmax scale * log2(e)
+};
+
+struct SegInfo {
+    int kind;        // 0 prefix, 1 private
+    int kvh, rb, b;  // b = -1 for prefix
+    int n_rows;      // valid rows in this row block
+    int row0;        // first stacked row of the block (prefix: in [0, N*nr); private: in [0, nr))
+    int tile_begin;  // global index of the segment's first tile
+    int n_tiles;
+    int tok_begin;   // logical token of the segment's first key (0 for prefix, P for private)
+    int n_tokens;    // keys in the segment (P or L_b)
+};
+
+__host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// cum[b] = tiles of branches < b (per private segment of that branch), cum[N] = sum.
+// Must be called by all threads of the block; cum lives in shared memory (N+1 ints).
+__device__ inline void build_branch_tile_prefix(const AttnParams& p, int* cum) {
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int b = 0; b < p.N; ++b) {
+            cum[b] = run;
+            int L = p.branch_lens[b];
+            L = L < 0 ? 0 : L;
+            run += ceil_div(L, p.tile_tokens);
+        }
+        cum[p.N] = run;
+    }
+    __syncthreads();
+}
+
+__device__ inline int total_tiles(const AttnParams& p, const int* cum) {
+    return p.n_pre * p.tiles_pre + p.Hkv * p.n_rb_priv * cum[p.N];
+}
+
+// Segment that contains global tile g (0 <= g < total).
+__device__ inline SegInfo segment_of_tile(const AttnParams& p, const int* cum, int g) {
+    SegInfo s;
+    const int pre_total = p.n_pre * p.tiles_pre;
+    if (g < pre_total) {
+        const int idx = g / p.tiles_pre;
+        s.kind = 0; s.b = -1;
+        s.kvh = idx / p.n_rb_pre; s.rb = idx % p.n_rb_pre;
+        s.row0 = s.rb * p.rb_rows;
+        s.n_rows = min(p.rb_rows, p.N * p.nr - s.row0);
+        s.tile_begin = idx * p.tiles_pre; s.n_tiles = p.tiles_pre;
+        s.tok_begin = 0; s.n_tokens = p.P;
+        return s;
+    }
+    const int per = p.Hkv * p.n_rb_priv;
+    const int gp = g - pre_total;
+    int lo = 0, hi = p.N - 1;                  // largest b with per*cum[b] <= gp
+    while (lo < hi) {
+        int mid = (lo + hi + 1) >> 1;
+        if (per * cum[mid] <= gp) lo = mid; else hi = mid - 1;
+    }
+    const int b = lo;
+    const int tb = cum[b + 1] - cum[b];
+    const int within = (gp - per * cum[b]) / tb;      // (kvh, rb) index inside the branch
+    s.kind = 1; s.b = b;
+    s.kvh = within / p.n_rb_priv; s.rb = within % p.n_rb_priv;
+    s.row0 = s.rb * p.rb_rows;
+    s.n_rows = min(p.rb_rows, p.nr - s.row0);
+    s.tile_begin = pre_total + per * cum[b] + within * tb; s.n_tiles = tb;
+    s.tok_begin = p.P; s.n_tokens = p.branch_lens[b];
+    return s;
+}
+
+__device__ inline int segment_index(const AttnParams& p, const SegInfo& s) {
+    return s.kind == 0 ? s.kvh * p.n_rb_pre + s.rb
+                       : p.n_pre + (s.b * p.Hkv + s.kvh) * p.n_rb_priv + s.rb;
+}
+
+// Where the piece (segment s, CTA c) keeps its partial result.
+__device__ inline void piece_slot(const AttnParams& p, const SegInfo& s, int cta, float*& o,
+                                  float2*& ml) {
+    if (s.kind == 0) {
+        const size_t id = (size_t)(s.kvh * p.n_rb_pre + s.rb) + cta;
+        o = p.part_o_pre + id * p.pre_stride * kHeadDim;
+        ml = p.part_ml_pre + id * p.pre_stride;
+    } else {
+        const size_t id = (size_t)((s.b * p.Hkv + s.kvh) * p.n_rb_priv + s.rb) + cta;
+        o = p.part_o_priv + id * p.priv_stride * kHeadDim;
+        ml = p.part_ml_priv + id * p.priv_stride;
+    }
+}
+
+// 64-bit visibility mask of query position i over the last R private tokens of its branch:
+// bit a set <=> row i sees token (L - R + a).  Causal: bits 0..i.  Tree: i and its ancestors.
+__device__ inline unsigned long long row_visibility(const AttnParams& p, int b, int i) {
+    if (p.tree_parents == nullptr) return i >= 63 ? ~0ull : ((2ull << i) - 1ull);
+    unsigned long long m = 0;
+    int a = i;
+    for (int guard = 0; a >= 0 && guard < kMaxTreeRows; ++guard) {
+        m |= 1ull << a;
+        int par = p.tree_parents[b * p.R + a];
+        a = par < a ? par : -1;               // malformed parents end the walk
+    }
+    return m;
+}
+
+struct Ctx {
+    tts_config cfg;
+    int device;
+    int n_sms;
+    cudaStream_t stream;
+    int last_cuda_error;
+    long long launches;
+    int32_t* d_status;
+    // split-KV workspace
+    float* part_o_pre; float2* part_ml_pre; float* part_o_priv; float2* part_ml_priv;
+    size_t pre_rows, priv_rows;       // allocated partial rows (each 128 fp32 + one float2)
+    // staging for the host entry point
+    void* stage; size_t stage_bytes;
+    void* tmap_cache;                  // opaque: tensor maps keyed by pool pointer
+    // profiling aid
+    int profiling, prof_n;
+    cudaEvent_t* prof_ev;              // 3 events per recorded call
+};
+constexpr int kProfMaxCalls = 4096;
+
+// kernel launchers (each returns the cudaError_t of its launch)
+cudaError_t launch_attn_simt(const AttnParams& p, cudaStream_t st);
+cudaError_t launch_attn_combine(const AttnParams& p, cudaStream_t st);
+cudaError_t launch_accept(const float* p_target, const float* q_draft, const int32_t* draft_tokens,
+                          const float* uniforms, int n_branches, int gamma, int vocab,
+                          int32_t* accepted_len, int32_t* next_token, int32_t* status,
+                          cudaStream_t st);
+int simt_rb_rows(int nr);
+constexpr int kSimtTileTokens = 64;
+
+// tcgen05 path
+constexpr int kUmmaRows = 128;         // MMA tile height = rows per row block
+constexpr int kUmmaTileTokens = 128;
+constexpr int kUmmaMinRows = 9;        // below this many stacked rows per KV head the CUDA-core kernel runs
+bool umma_available();
+cudaError_t launch_attn_umma(Ctx* c, const AttnParams& p, cudaStream_t st);
+void umma_release(Ctx* c);
+
+}  // namespace tts

@@ -1,0 +1,192 @@
+"""Parity of the CUDA attention path against the CPU oracle, through the C-ABI.
+Tolerance (north-star): |gpu - oracle| <= 1e-2 + 1e-2 |oracle| per element for bf16 inputs with
+fp32 accumulation; because that band is loose on N(0,1) data, every case is also gated on the
+relative RMS error and there are sentinel / peaky-softmax cases whose errors would be O(1)."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2505_19634_b200 as tts
+import tts_inputs as ti
+from gpu_harness import ATTN_IMPLS, IMPL_NAMES, assert_attn_close, attn_errors, make_ctx, run_attn
+
+pytestmark = pytest.mark.gpu
+
+impl_param = pytest.mark.parametrize("impl", ATTN_IMPLS, ids=lambda i: IMPL_NAMES[i])
+
+
+def oracle_out(case, **kw):
+    return oracle.verify_attn(case.q, case.k_pages, case.v_pages, case.block_table, case.prefix_len,
+                              case.branch_lens, case.shape.gamma, **kw)
+
+
+def bf16_round(x):
+    return ti.bf16_bits_to_f32(ti.f32_to_bf16_bits(x.astype(np.float32))).astype(np.float64)
+
+
+@impl_param
+def test_tiny_config(impl):
+    case = ti.make_attn_case(ti.CONFIGS["tiny"], 0x5EED)
+    want = oracle_out(case)
+    got = run_attn(case, impl)
+    assert_attn_close(got, want, what="tiny")
+    got32 = run_attn(case, impl, out_dtype=tts.OUT_FP32)
+    assert attn_errors(got32, want)[1] < 4e-3          # only the bf16 rounding of P (tensor path) remains
+    # bf16 output = round-to-nearest-even of the fp32 result
+    assert np.array_equal(got, bf16_round(got32))
+
+
+@impl_param
+def test_3b_config(impl):
+    case = ti.make_attn_case(ti.CONFIGS["3b"], 0x5EED + 1)
+    ti.poison_unused_slots(case)
+    assert_attn_close(run_attn(case, impl), oracle_out(case), what="3b")
+
+
+SMALL = ti.AttnShape("small", n_q_heads=8, n_kv_heads=2, prefix_len=48, n_branches=3, gamma=2,
+                     branch_lens=(19, 3, 140), permute_pages=True, extra_pages=5)
+
+EDGE_SHAPES = {
+    "ragged": SMALL,
+    "no_prefix": replace(SMALL, prefix_len=0),
+    "gamma0": replace(SMALL, gamma=0, branch_lens=(1, 16, 17)),
+    "min_len": replace(SMALL, gamma=3, branch_lens=(4, 4, 4)),
+    "one_branch": replace(SMALL, n_branches=1, branch_lens=(300,), gamma=4),
+    "mha": replace(SMALL, n_q_heads=4, n_kv_heads=4),
+    "group8_gamma5": replace(SMALL, n_q_heads=16, n_kv_heads=2, gamma=5, branch_lens=(6, 130, 257)),
+    "page_multiple": replace(SMALL, branch_lens=(16, 128, 256), prefix_len=128),
+    "long_prefix_short_private": replace(SMALL, prefix_len=640, branch_lens=(3, 5, 9)),
+    "many_branches": replace(SMALL, n_branches=33, gamma=1, branch_lens=tuple(2 + 7 * i for i in range(33))),
+    "tile_straddle": replace(SMALL, gamma=5, branch_lens=(130, 131, 258)),   # draft rows cross a 128-token tile edge
+}
+
+
+@impl_param
+@pytest.mark.parametrize("name", list(EDGE_SHAPES))
+def test_edge_shapes(impl, name):
+    case = ti.make_attn_case(EDGE_SHAPES[name], 77)
+    ti.poison_unused_slots(case)               # NaN wherever no query may look
+    assert_attn_close(run_attn(case, impl), oracle_out(case), what=name)
+
+
+@impl_param
+def test_sentinel_in_masked_positions(impl):
+    """Enormous K/V in every position a row must not see: one leaked key changes out by O(1)."""
+    shp = replace(SMALL, gamma=3, branch_lens=(19, 4, 140))
+    case = ti.make_attn_case(shp, 5)
+    clean = oracle_out(case)
+    big = ti.f32_to_bf16_bits(np.array([3.0e4], np.float32))[0]
+    for b in range(shp.n_branches):
+        L = int(case.branch_lens[b])
+        page, slot = ti.token_slot(case, b, case.prefix_len + L - 1)     # visible to the last row only
+        case.k_pages[page, :, slot, :] = big
+        case.v_pages[page, :, slot, :] = big
+    ti.poison_unused_slots(case, bits=int(big))
+    want = oracle_out(case)
+    assert np.array_equal(want[:, :3], clean[:, :3])
+    got = run_attn(case, impl)
+    assert_attn_close(got[:, :3], want[:, :3], what="rows that must not see the sentinel")
+
+
+@impl_param
+def test_peaky_softmax(impl):
+    """Queries scaled by 8: the softmax concentrates on a few keys and masking/ordering errors show."""
+    case = ti.make_attn_case(replace(SMALL, branch_lens=(200, 77, 140)), 9, q_scale=8.0)
+    want = oracle_out(case)
+    got = run_attn(case, impl)
+    assert_attn_close(got, want, rms_gate=8e-3, what="peaky")
+
+
+@impl_param
+def test_rescale_path_with_growing_scores(impl):
+    """Keys whose scores grow along the sequence force the running max to move in every tile."""
+    shp = replace(SMALL, n_branches=2, branch_lens=(700, 390), prefix_len=256, gamma=3)
+    case = ti.make_attn_case(shp, 21)
+    kf = ti.bf16_bits_to_f32(case.k_pages)
+    qf = ti.bf16_bits_to_f32(case.q)
+    qf[..., 0] = 4.0
+    case.q = ti.f32_to_bf16_bits(qf)
+    for b in range(2):
+        total = case.prefix_len + int(case.branch_lens[b])
+        for t in range(total):
+            page, slot = ti.token_slot(case, b, t)
+            kf[page, :, slot, 0] = 0.08 * t          # score contribution 4*0.08*t/sqrt(128) ~ 0.028 t
+    case.k_pages = ti.f32_to_bf16_bits(kf)
+    assert_attn_close(run_attn(case, impl), oracle_out(case), rms_gate=8e-3, what="growing scores")
+
+
+@impl_param
+def test_page_permutation_invariance(impl):
+    shp = replace(SMALL, permute_pages=False, extra_pages=0)
+    a = ti.make_attn_case(shp, 11)
+    perm = np.random.default_rng(0).permutation(a.num_pages)
+    inv = np.argsort(perm)
+    b = ti.make_attn_case(shp, 11)
+    b.k_pages = np.ascontiguousarray(a.k_pages[perm]); b.v_pages = np.ascontiguousarray(a.v_pages[perm])
+    b.block_table = np.where(a.block_table >= 0, inv[np.maximum(a.block_table, 0)], -1).astype(np.int32)
+    assert np.array_equal(run_attn(a, impl), run_attn(b, impl))
+
+
+@impl_param
+def test_tree_mask(impl):
+    shp = replace(SMALL, gamma=11, branch_lens=(19, 12, 140))
+    case = ti.make_attn_case(shp, 31)
+    parents = ti.make_tree_parents(3, 12, 4, seed=8)
+    want = oracle_out(case, mask_kind=1, tree_parents=parents)
+    got = run_attn(case, impl, tree_parents=parents)
+    assert_attn_close(got, want, what="tree")
+    chain = np.tile(np.arange(-1, 11, dtype=np.int32), (3, 1))
+    assert np.array_equal(run_attn(case, impl, tree_parents=chain), run_attn(case, impl))
+
+
+@impl_param
+def test_sweep_points(impl):
+    """A few points of the branch/length sweep at reduced lengths (full shapes: Hq 40 / Hkv 8)."""
+    for n, g, seed in ((1, 1, 1), (4, 5, 2), (16, 3, 3)):
+        shp = ti.sweep_shape(n, g, seed, lo=40, hi=600)
+        case = ti.make_attn_case(shp, seed)
+        ti.poison_unused_slots(case)
+        assert_attn_close(run_attn(case, impl), oracle_out(case), what=shp.name)
+
+
+def test_context_reuse_and_launch_count():
+    case = ti.make_attn_case(SMALL, 3)
+    ctx = make_ctx(case, max_rows=6, max_branches=8)
+    a = run_attn(case, ctx=ctx)
+    n1 = ctx.tts_launch_count()
+    b = run_attn(case, ctx=ctx)
+    assert np.array_equal(a, b)
+    assert n1 >= 2 and ctx.tts_launch_count() == 2 * n1
+    ctx.close()
+
+
+def test_argument_errors_are_status_codes():
+    import torch
+    case = ti.make_attn_case(SMALL, 3)
+    ctx = make_ctx(case)
+    z = torch.zeros(64, device="cuda", dtype=torch.int32)
+    for kw, want in ((dict(prefix_len=8), -1), (dict(n_branches=0), -1), (dict(n_branches=99), -1),
+                     (dict(gamma=-1), -1), (dict(gamma=40), -1), (dict(mask_kind=1), -2), (dict(mask_kind=7), -2)):
+        args = dict(prefix_len=48, n_branches=3, gamma=2, mask_kind=0)
+        args.update(kw)
+        with pytest.raises(tts.TtsError) as ei:
+            ctx.tts_verify_attn(z, z, z, z, args["prefix_len"], z, args["n_branches"], args["gamma"],
+                                args["mask_kind"], z)
+        assert ei.value.status == want, kw
+    with pytest.raises(tts.TtsError):
+        ctx.tts_verify_attn(None, z, z, z, 48, z, 3, 2, 0, z)
+    with pytest.raises(tts.TtsError):                   # misaligned q
+        ctx.tts_verify_attn(z.data_ptr() + 4, z, z, z, 48, z, 3, 2, 0, z)
+    ctx.close()
+
+
+def test_debug_bounds_reports_bad_page_id_without_faulting():
+    case = ti.make_attn_case(SMALL, 3)
+    case.block_table[1, 3] = case.num_pages + 1000        # out-of-range page of branch 1
+    ctx = make_ctx(case, impl=tts.ATTN_SIMT, debug=True)
+    run_attn(case, ctx=ctx, check_status=False)
+    assert ctx.tts_last_status() == -4
+    assert ctx.tts_last_status() == 0                     # reading clears it
+    ctx.close()
