@@ -38,11 +38,14 @@ __global__ void __launch_bounds__(kRowsPerBlock * 32) attn_combine_kernel(const 
     float m_run = -INFINITY, l_run = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 
-    auto merge = [&](const float* o_base, const float2* ml_base, int stride, int seg_local, int r,
-                     int t_begin, int n_tiles) {
+    // rows of one piece: `n_copies` stacked blocks of `rows_in_block` rows; row r of every block
+    // belongs to this output row
+    auto merge = [&](const float* o_base, const float2* ml_base, int stride, int seg_local, int r0,
+                     int rows_in_block, int n_copies, int t_begin, int n_tiles) {
         if (n_tiles <= 0) return;
         const int c0 = t_begin / tpc, c1 = (t_begin + n_tiles - 1) / tpc;
-        for (int c = c0; c <= c1; ++c) {
+        for (int cc = c0 * n_copies; cc < (c1 + 1) * n_copies; ++cc) {
+            const int c = cc / n_copies, r = (cc % n_copies) * rows_in_block + r0;
             const size_t id = (size_t)seg_local + c;
             const float2 ml = ml_base[id * stride + r];
             if (!(ml.y > 0.f)) continue;                  // piece saw no visible key for this row
@@ -63,13 +66,14 @@ __global__ void __launch_bounds__(kRowsPerBlock * 32) attn_combine_kernel(const 
         const int pr = b * p.nr + r_priv;
         const int rb = pr / p.rb_rows, r = pr % p.rb_rows;
         const int seg = kvh * p.n_rb_pre + rb;
-        merge(p.part_o_pre, p.part_ml_pre, p.pre_stride, seg, r, seg * p.tiles_pre, p.tiles_pre);
+        merge(p.part_o_pre, p.part_ml_pre, p.pre_stride, seg, r, 0, 1, seg * p.tiles_pre, p.tiles_pre);
     }
     {
         const int rb = r_priv / p.rb_rows, r = r_priv % p.rb_rows;
         const int within = kvh * p.n_rb_priv + rb;
         const int seg = b * per + within;
-        merge(p.part_o_priv, p.part_ml_priv, p.priv_stride, seg, r, pre_total + per * before + within * tiles_b, tiles_b);
+        merge(p.part_o_priv, p.part_ml_priv, p.priv_stride, seg, r, min(p.rb_rows, p.nr - rb * p.rb_rows), p.copies,
+              pre_total + per * before + within * tiles_b, tiles_b);
     }
 
     const float inv = l_run > 0.f ? 1.f / l_run : 0.f;

@@ -1,8 +1,606 @@
-// tcgen05 verify attention (placeholder until the tensor-core kernel lands).
+// Tensor-core verify attention for sm_100a: tcgen05.mma with TMEM accumulators, K/V page tiles
+// staged by TMA, fp32 online softmax between the two contractions.
+//
+// One persistent CTA per SM walks its run of the global tile list (tts_internal.cuh).  A tile is
+// 128 KV tokens of one KV head = 8 pages gathered through the block table, each page-head tile
+// (16 tokens x 128 dims, 4 KiB contiguous) arriving as two 128-byte-swizzled TMA boxes.
+//
+//   warp 4      producer: per tile, arms the K and V "full" barriers with the byte count and
+//               issues the TMA boxes (K ring and V ring, 2 slots x 32 KiB each)
+//   warp 5      MMA issuer (one thread): S = Q K^T into one of two TMEM buffers, then
+//               O (+)= P V once the softmax warps have published P; frees ring slots with
+//               tcgen05.commit
+//   warps 0-3   softmax: thread = TMEM lane = query row.  Reads S, keeps the running max m and
+//               sum l in fp32, writes P (bf16, swizzled K-major) to shared memory for the second
+//               contraction, rescales O in TMEM only when the max moved by more than 2^8
+//               (the final result is exact either way, l carries the same reference), and
+//               writes the piece's partial (m, l, O) at the end.
+//
+// Few query rows per KV head (nr = (gamma+1) * G, e.g. 20) would leave most of the 128-row MMA
+// tile idle, so the rows of a private segment are replicated `copies` = 2 or 4 times along M and
+// copy c only looks at its own 128/copies-column slice of every S tile: the softmax work per
+// thread shrinks by `copies`, no cross-thread reduction is needed (each copy is an independent
+// split of the keys with its own m and l), and the merge kernel folds the copies together with
+// the pieces.  The MMA cost is unchanged (M is 128 regardless).
+//
+// Every wait is bounded: when a limit runs out the CTA raises TTS_ERR_DEVICE_TIMEOUT in the
+// status word, all roles leave their loops, in-flight copies are awaited (bounded) and TMEM is
+// released before the CTA returns.
+#include <cuda.h>
+
+#include <vector>
+
 #include "tts_internal.cuh"
 
 namespace tts {
-bool umma_available() { return false; }
-cudaError_t launch_attn_umma(Ctx*, const AttnParams&, cudaStream_t) { return cudaErrorNotSupported; }
-void umma_release(Ctx*) {}
+
+namespace {
+
+constexpr int kTile = kUmmaTileTokens;            // 128 tokens
+constexpr int kRows = kUmmaRows;                   // 128 = MMA M
+constexpr int kThreadsUmma = 192;
+constexpr int kHalfBytes = kRows * 128;            // one 64-element K-block of a 128-row operand: 16 KiB
+constexpr int kOperandBytes = 2 * kHalfBytes;      // 32 KiB
+constexpr int kRing = 2;
+constexpr uint32_t kTmemCols = 512;
+constexpr long long kWaitLimitNs = 400ll * 1000 * 1000;
+
+// shared memory map (offsets from a 1024-byte aligned base)
+constexpr int kOffQ = 0;
+constexpr int kOffP = kOffQ + kOperandBytes;
+constexpr int kOffK = kOffP + kOperandBytes;
+constexpr int kOffV = kOffK + kRing * kOperandBytes;
+constexpr int kOffBar = kOffV + kRing * kOperandBytes;        // 196608
+constexpr int kNumBars = 16;
+constexpr int kOffMisc = kOffBar + kNumBars * 8;
+constexpr int kOffCum = kOffMisc + 64;
+constexpr int kUmmaMaxBranches = 1024;
+constexpr int kSmemBytes = kOffCum + (kUmmaMaxBranches + 1) * 4 + 1024;   // + slack for manual alignment
+
+enum Bar { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, S_FULL = 8, S_FREE = 10, P_FULL = 12, PV_DONE = 13, Q_FULL = 14 };
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ long long global_ns() {
+    long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+struct Abort {
+    volatile int* flag;     // shared: set when any wait of this CTA ran out
+    int32_t* status;        // global status word
+};
+
+// Bounded wait.  Returns false if the CTA is aborting (this or another wait ran out of time).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = global_ns();
+    for (int spin = 0;; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 63) == 63) {
+            if (*ab.flag) return false;
+            if (global_ns() - t0 > kWaitLimitNs) {
+                *ab.flag = 1;
+                atomicMin(ab.status, (int)TTS_ERR_DEVICE_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).
+//   K-major operand  (rows x 64-element K-block, 128-byte rows): lbo = 16, sbo = 1024 (8-row atoms)
+//   MN-major operand (64-element MN-block x K rows):             lbo = bytes between MN-blocks,
+//                                                                 sbo = 1024 (8 K-rows)
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(lbo_bytes >> 4) << 16;
+    d |= (uint64_t)(sbo_bytes >> 4) << 32;
+    d |= 1ull << 46;                      // descriptor version
+    d |= 2ull << 61;                      // SWIZZLE_128B
+    return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128; B either K-major or MN-major.
+__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// byte offset of the 16-byte chunk holding elements [8*chunk, 8*chunk+8) of `row` in a 128-row,
+// 128-element-wide K-major operand with 128-byte swizzle
+__device__ __forceinline__ uint32_t kmajor_chunk_off(int row, int chunk) {
+    return (uint32_t)((chunk >> 3) * kHalfBytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+}
+
+struct PieceWalk {                    // every role iterates the CTA's pieces the same way
+    int g, g_end;
+};
+
+__global__ void __launch_bounds__(kThreadsUmma, 1)
+attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v) {
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = sbase + kOffBar;
+    auto bar = [&](int i) { return bar0 + 8u * i; };
+    volatile int* misc = reinterpret_cast<volatile int*>(smem + kOffMisc);   // [0] abort flag, [1] tmem base
+    int* cum = reinterpret_cast<int*>(smem + kOffCum);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const Abort ab{misc, p.status};
+
+    build_branch_tile_prefix(p, cum);
+    const int total = total_tiles(p, cum);
+    const int tpc = ceil_div(total, p.grid);
+    const int g_begin = blockIdx.x * tpc;
+    const int g_end = min(total, g_begin + tpc);
+    if (g_begin >= g_end) return;                          // uniform: nothing to do for this CTA
+
+    // ---- set-up: zero P and the V ring (nothing non-finite may ever meet a zero weight), barriers, TMEM ----
+    for (int i = tid; i < (kOperandBytes + kRing * kOperandBytes) / 16; i += kThreadsUmma) {
+        const int off = i * 16 < kOperandBytes ? kOffP + i * 16 : kOffV + (i * 16 - kOperandBytes);
+        *reinterpret_cast<uint4*>(smem + off) = make_uint4(0, 0, 0, 0);
+    }
+    if (tid == 0) {
+        misc[0] = 0;
+        for (int i = 0; i < kRing; ++i) {
+            mbar_init(bar(K_FULL + i), 1); mbar_init(bar(K_EMPTY + i), 1);
+            mbar_init(bar(V_FULL + i), 1); mbar_init(bar(V_EMPTY + i), 1);
+            mbar_init(bar(S_FULL + i), 1); mbar_init(bar(S_FREE + i), 128);
+        }
+        mbar_init(bar(P_FULL), 128); mbar_init(bar(PV_DONE), 1); mbar_init(bar(Q_FULL), 128);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + kOffMisc + 4), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = (uint32_t)misc[1];
+    const uint32_t tmem_s[2] = {tmem, tmem + 128u};
+    const uint32_t tmem_o = tmem + 256u;
+
+    if (warp == 4) {
+        // =========================== producer ===========================
+        int it = 0;                                         // tiles issued by this CTA
+        int g = g_begin;
+        bool alive = true;
+        while (g < g_end && alive) {
+            const SegInfo seg = segment_of_tile(p, cum, g);
+            const int t_first = g - seg.tile_begin, t_last = min(seg.n_tiles, g_end - seg.tile_begin);
+            const int32_t* bt = p.block_table + (size_t)(seg.kind == 0 ? 0 : seg.b) * p.max_blocks;
+            for (int t = t_first; t < t_last && alive; ++t, ++it) {
+                const int slot = it % kRing;
+                const uint32_t par = ((it / kRing) & 1) ^ 1;
+                const int tok0 = t * kTile;
+                const int n_pages = ceil_div(min(kTile, seg.n_tokens - tok0), kPage);
+                int page = 0;
+                if (lane < n_pages) {
+                    page = bt[(seg.tok_begin + tok0) / kPage + lane];
+                    if (p.debug && (page < 0 || page >= p.num_pages)) {
+                        atomicMin(p.status, (int)TTS_ERR_DEVICE_BOUNDS);
+                        page = 0;
+                    }
+                }
+                const int y = (page * p.Hkv + seg.kvh) * kPage;
+                // K
+                if (lane == 0) {
+                    alive = mbar_wait(bar(K_EMPTY + slot), par, ab);
+                    if (alive) mbar_arrive_expect_tx(bar(K_FULL + slot), (uint32_t)n_pages * 4096u);
+                }
+                alive = __shfl_sync(0xffffffffu, alive, 0);
+                if (!alive) break;
+                if (lane < n_pages) {
+                    const uint32_t dst = sbase + kOffK + slot * kOperandBytes + lane * 2048;
+                    tma_load_2d(dst, &tm_k, 0, y, bar(K_FULL + slot));
+                    tma_load_2d(dst + kHalfBytes, &tm_k, 64, y, bar(K_FULL + slot));
+                }
+                // V
+                if (lane == 0) {
+                    alive = mbar_wait(bar(V_EMPTY + slot), par, ab);
+                    if (alive) mbar_arrive_expect_tx(bar(V_FULL + slot), (uint32_t)n_pages * 4096u);
+                }
+                alive = __shfl_sync(0xffffffffu, alive, 0);
+                if (!alive) break;
+                if (lane < n_pages) {
+                    const uint32_t dst = sbase + kOffV + slot * kOperandBytes + lane * 2048;
+                    tma_load_2d(dst, &tm_v, 0, y, bar(V_FULL + slot));
+                    tma_load_2d(dst + kHalfBytes, &tm_v, 64, y, bar(V_FULL + slot));
+                }
+            }
+            g = seg.tile_begin + t_last;
+        }
+        // Copies this warp started must have landed before the CTA may exit: the consumers wait on
+        // the same phases in the normal case; after an abort wait for them here (bounded).
+        if (*ab.flag && lane == 0) {
+            for (int back = 1; back <= kRing && back <= it; ++back) {
+                const int j = it - back;
+                const Abort quiet{misc + 2, p.status};       // do not re-raise; misc[2] is scratch
+                misc[2] = 0;
+                mbar_wait(bar(K_FULL + j % kRing), (j / kRing) & 1, quiet);
+                mbar_wait(bar(V_FULL + j % kRing), (j / kRing) & 1, quiet);
+            }
+        }
+    } else if (warp == 5) {
+        // =========================== MMA issuer ===========================
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
+            int it = 0, piece = 0;
+            int g = g_begin;
+            bool alive = true;
+            auto issue_qk = [&](int j) -> bool {
+                const int slot = j % kRing, sb = j & 1;
+                if (!mbar_wait(bar(K_FULL + slot), (j / kRing) & 1, ab)) return false;
+                if (!mbar_wait(bar(S_FREE + sb), ((j >> 1) & 1) ^ 1, ab)) return false;
+                tc_fence_after();
+                const uint32_t qa = sbase + kOffQ, ka = sbase + kOffK + slot * kOperandBytes;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                    umma_bf16(tmem_s[sb], smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), idesc_qk, ks > 0);
+                }
+                umma_commit(bar(K_EMPTY + slot));
+                umma_commit(bar(S_FULL + sb));
+                return true;
+            };
+            while (g < g_end && alive) {
+                const SegInfo seg = segment_of_tile(p, cum, g);
+                const int t_first = g - seg.tile_begin, t_last = min(seg.n_tiles, g_end - seg.tile_begin);
+                const int n = t_last - t_first;
+                alive = mbar_wait(bar(Q_FULL), piece & 1, ab);
+                if (!alive) break;
+                tc_fence_after();
+                alive = issue_qk(it);
+                for (int j = 0; j < n && alive; ++j) {
+                    if (j + 1 < n) { alive = issue_qk(it + j + 1); if (!alive) break; }
+                    const int cur = it + j, slot = cur % kRing;
+                    alive = mbar_wait(bar(P_FULL), cur & 1, ab) && mbar_wait(bar(V_FULL + slot), (cur / kRing) & 1, ab);
+                    if (!alive) break;
+                    tc_fence_after();
+                    const uint32_t pa = sbase + kOffP, va = sbase + kOffV + slot * kOperandBytes;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t aoff = (ks >> 2) * kHalfBytes + (ks & 3) * 32;      // P: K-major over tokens
+                        const uint32_t boff = ks * 2048;                                    // V: 16 token rows per step
+                        umma_bf16(tmem_o, smem_desc(pa + aoff, 16, 1024), smem_desc(va + boff, kHalfBytes, 1024), idesc_pv,
+                                  (j > 0 || ks > 0) ? 1u : 0u);
+                    }
+                    umma_commit(bar(V_EMPTY + slot));
+                    umma_commit(bar(PV_DONE));
+                }
+                it += n; ++piece;
+                g = seg.tile_begin + t_last;
+            }
+        }
+    } else {
+        // =========================== softmax warps ===========================
+        const int L = tid;                                  // TMEM lane = row of the MMA tile
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        int it = 0;
+        int g = g_begin;
+        bool alive = true;
+        while (g < g_end && alive) {
+            const SegInfo seg = segment_of_tile(p, cum, g);
+            const int t_first = g - seg.tile_begin, t_last = min(seg.n_tiles, g_end - seg.tile_begin);
+            const int ncopy = seg.kind == 0 ? 1 : p.copies;
+            const int rpc = kRows / ncopy;                   // TMEM lanes per copy
+            const int W = kTile / ncopy;                     // S columns this thread looks at
+            const int copy = L / rpc, r = L % rpc;
+            const bool valid = r < seg.n_rows;
+            const int col0 = copy * W;
+
+            // ---- stage Q (replicated per copy, zero rows elsewhere), per-row mask ----
+            unsigned long long vis = ~0ull;
+            {
+                const __nv_bfloat16* src = nullptr;
+                if (valid) {
+                    int row = seg.row0 + r, b = seg.b;
+                    if (seg.kind == 0) { b = row / p.nr; row = row % p.nr; }
+                    const int i = row / p.G, gq = row % p.G;
+                    src = p.q + (((size_t)b * p.R + i) * p.Hq + seg.kvh * p.G + gq) * kHeadDim;
+                    if (seg.kind == 1) vis = row_visibility(p, b, i);
+                }
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (valid) v = __ldg(reinterpret_cast<const uint4*>(src) + c);
+                    *reinterpret_cast<uint4*>(smem + kOffQ + kmajor_chunk_off(L, c)) = v;
+                }
+            }
+            fence_proxy_async();
+            mbar_arrive(bar(Q_FULL));
+
+            float m_ref = -INFINITY, l_sum = 0.f;           // reference max (log2 units) and running sum
+            const int Ltok = seg.n_tokens;
+            const int tail0 = seg.kind == 1 ? Ltok - p.R : Ltok;     // first token that needs the row mask
+
+            for (int t = t_first; t < t_last && alive; ++t, ++it) {
+                const int sb = it & 1;
+                const int tok0 = t * kTile;
+                const bool need_mask = tok0 + kTile > tail0;        // uniform: tile touches masked / missing tokens
+                alive = __all_sync(0xffffffffu, mbar_wait(bar(S_FULL + sb), (it >> 1) & 1, ab));
+                if (!alive) break;
+                tc_fence_after();
+                const uint32_t s_addr = tmem_s[sb] + lane_base + (uint32_t)col0;
+
+                auto allowed = [&](int col) -> bool {       // col = column inside the tile
+                    const int j = tok0 + col;
+                    if (j >= Ltok) return false;
+                    if (j >= tail0) return (vis >> (j - tail0)) & 1ull;
+                    return true;
+                };
+
+                // pass 1: row max over this thread's columns
+                float mx = -INFINITY;
+                for (int ch = 0; ch < W / 32; ++ch) {
+                    uint32_t sv[32];
+                    tmem_ld32(s_addr + 32u * ch, sv);
+                    tmem_wait_ld();
+                    if (need_mask) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (allowed(col0 + 32 * ch + c)) mx = fmaxf(mx, __uint_as_float(sv[c]));
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(sv[c]));
+                    }
+                }
+                mx *= p.scale_log2;                          // scale > 0; -inf stays -inf
+                const bool move = mx > m_ref + 8.f || (m_ref == -INFINITY && mx > -INFINITY);
+                const float m_new = move ? mx : m_ref;
+                const float factor = (move && m_ref != -INFINITY) ? ex2(m_ref - m_new) : 1.f;
+
+                // the previous tile's P.V must be finished before P is overwritten or O touched
+                if (it > 0) {
+                    alive = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE), (it - 1) & 1, ab));
+                    if (!alive) break;
+                    tc_fence_after();
+                }
+                if (t > t_first && __any_sync(0xffffffffu, factor != 1.f)) {
+                    for (int ch = 0; ch < 4; ++ch) {
+                        uint32_t ov[32];
+                        tmem_ld32(tmem_o + lane_base + 32u * ch, ov);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * factor);
+                        tmem_st32(tmem_o + lane_base + 32u * ch, ov);
+                    }
+                    tmem_wait_st();
+                }
+                l_sum *= factor;
+                m_ref = m_new;
+
+                // pass 2: probabilities -> P (bf16) in shared memory
+                const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+                for (int ch = 0; ch < W / 32; ++ch) {
+                    uint32_t sv[32];
+                    tmem_ld32(s_addr + 32u * ch, sv);
+                    tmem_wait_ld();
+                    float pr[32];
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        float e = ex2(fmaf(__uint_as_float(sv[c]), p.scale_log2, neg_m));
+                        if (need_mask && !allowed(col0 + 32 * ch + c)) e = 0.f;
+                        pr[c] = e;
+                        l_sum += e;
+                    }
+                    const int tc0 = col0 + 32 * ch;          // first token column of this chunk
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint4 pk;
+                        __nv_bfloat162 h0 = __floats2bfloat162_rn(pr[8 * q4 + 0], pr[8 * q4 + 1]);
+                        __nv_bfloat162 h1 = __floats2bfloat162_rn(pr[8 * q4 + 2], pr[8 * q4 + 3]);
+                        __nv_bfloat162 h2 = __floats2bfloat162_rn(pr[8 * q4 + 4], pr[8 * q4 + 5]);
+                        __nv_bfloat162 h3 = __floats2bfloat162_rn(pr[8 * q4 + 6], pr[8 * q4 + 7]);
+                        pk.x = *reinterpret_cast<uint32_t*>(&h0); pk.y = *reinterpret_cast<uint32_t*>(&h1);
+                        pk.z = *reinterpret_cast<uint32_t*>(&h2); pk.w = *reinterpret_cast<uint32_t*>(&h3);
+                        *reinterpret_cast<uint4*>(smem + kOffP + kmajor_chunk_off(L, (tc0 >> 3) + q4)) = pk;
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(bar(S_FREE + sb));               // S buffer may be overwritten
+
+                // last tile of a private segment: zero the V rows of the loaded pages past the branch end
+                if (need_mask) {
+                    const int n_valid = min(kTile, Ltok - tok0);
+                    const int n_loaded = ceil_div(n_valid, kPage) * kPage;
+                    if (n_valid < n_loaded) {
+                        const int slot = it % kRing;
+                        alive = __all_sync(0xffffffffu, mbar_wait(bar(V_FULL + slot), (it / kRing) & 1, ab));
+                        if (!alive) break;
+                        for (int idx = tid; idx < (n_loaded - n_valid) * 16; idx += 128) {
+                            const int row = n_valid + idx / 16, c = idx % 16;
+                            *reinterpret_cast<uint4*>(smem + kOffV + slot * kOperandBytes + (c >> 3) * kHalfBytes + row * 128 + ((c & 7) << 4)) =
+                                make_uint4(0, 0, 0, 0);
+                        }
+                    }
+                }
+                fence_proxy_async();
+                mbar_arrive(bar(P_FULL));
+            }
+            if (!alive) break;
+
+            // ---- piece epilogue: partial (m, l, O) ----
+            alive = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE), (it - 1) & 1, ab));
+            if (!alive) break;
+            tc_fence_after();
+            float* po; float2* pml;
+            piece_slot(p, seg, blockIdx.x, po, pml);
+            const int prow = copy * seg.n_rows + r;          // copies of a private piece are stacked
+            for (int ch = 0; ch < 4; ++ch) {
+                uint32_t ov[32];
+                tmem_ld32(tmem_o + lane_base + 32u * ch, ov);
+                tmem_wait_ld();
+                if (valid) {
+                    float4* dst = reinterpret_cast<float4*>(po + (size_t)prow * kHeadDim + 32 * ch);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        dst[c] = make_float4(__uint_as_float(ov[4 * c]), __uint_as_float(ov[4 * c + 1]),
+                                             __uint_as_float(ov[4 * c + 2]), __uint_as_float(ov[4 * c + 3]));
+                }
+            }
+            if (valid) pml[prow] = make_float2(m_ref, l_sum);
+            tc_fence_before();
+            g = seg.tile_begin + t_last;
+        }
+    }
+
+    // ---- teardown: everyone arrives here, normally or after an abort ----
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+struct MapEntry { const void* ptr; long rows; CUtensorMap map; };
+struct MapCache { std::vector<MapEntry> entries; };
+
+// 2-D view of a page pool: rows = num_pages * Hkv * 16 tokens of 128 bf16; box = 64 dims x 16 tokens.
+const CUtensorMap* pool_map(Ctx* c, const void* pool, cudaError_t* err) {
+    if (!c->tmap_cache) c->tmap_cache = new MapCache();
+    MapCache* mc = static_cast<MapCache*>(c->tmap_cache);
+    const long rows = (long)c->cfg.num_pages * c->cfg.n_kv_heads * kPage;
+    for (auto& e : mc->entries)
+        if (e.ptr == pool && e.rows == rows) return &e.map;
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) { *err = cudaErrorNotSupported; return nullptr; }
+    MapEntry e;
+    e.ptr = pool; e.rows = rows;
+    const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kPage};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(pool), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { *err = cudaErrorInvalidValue; return nullptr; }
+    if (mc->entries.size() >= 512) mc->entries.erase(mc->entries.begin());
+    mc->entries.push_back(e);
+    return &mc->entries.back().map;
+}
+
+}  // namespace
+
+bool umma_available() { return true; }
+
+int umma_copies(int nr) { return nr <= 32 ? 4 : (nr <= 64 ? 2 : 1); }
+
+cudaError_t launch_attn_umma(Ctx* c, const AttnParams& p, cudaStream_t st) {
+    if (p.N > kUmmaMaxBranches) return cudaErrorInvalidValue;
+    cudaError_t err = cudaSuccess;
+    const CUtensorMap* mk = pool_map(c, p.k_pages, &err);
+    if (!mk) return err;
+    const CUtensorMap mk_copy = *mk;                       // the cache may reallocate on the next insert
+    const CUtensorMap* mv = pool_map(c, p.v_pages, &err);
+    if (!mv) return err;
+    static bool attr_set[64] = {};                          // the attribute is per device
+    if (c->device < 0 || c->device >= 64 || !attr_set[c->device]) {
+        err = cudaFuncSetAttribute(attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (err != cudaSuccess) return err;
+        if (c->device >= 0 && c->device < 64) attr_set[c->device] = true;
+    }
+    attn_umma_kernel<<<p.grid, kThreadsUmma, kSmemBytes, st>>>(p, mk_copy, *mv);
+    return cudaGetLastError();
+}
+
+void umma_release(Ctx* c) {
+    delete static_cast<MapCache*>(c->tmap_cache);
+    c->tmap_cache = nullptr;
+}
+
 }  // namespace tts

@@ -43,7 +43,8 @@ struct AttnParams {
     int P;                          // prefix tokens
     int max_blocks, num_pages;
     int rb_rows;                    // rows per row block
-    int pre_stride, priv_stride;    // rows reserved per piece: min(rb_rows, N*nr) / min(rb_rows, nr)
+    int pre_stride, priv_stride;    // rows reserved per piece: min(rb_rows, N*nr) / copies * min(rb_rows, nr)
+    int copies;                     // tcgen05 path: independent key-slice copies of a private piece's rows
     int n_rb_pre, n_rb_priv;        // row blocks per prefix kv head / per (branch, kv head)
     int n_pre;                      // prefix segments (0 when P == 0)
     int tiles_pre;                  // tiles per prefix segment
@@ -187,6 +188,7 @@ constexpr int kUmmaRows = 128;         // MMA tile height = rows per row block
 constexpr int kUmmaTileTokens = 128;
 constexpr int kUmmaMinRows = 9;        // below this many stacked rows per KV head the CUDA-core kernel runs
 bool umma_available();
+int umma_copies(int nr);              // replication factor of a private piece's rows along the MMA M dimension
 cudaError_t launch_attn_umma(Ctx* c, const AttnParams& p, cudaStream_t st);
 void umma_release(Ctx* c);
 

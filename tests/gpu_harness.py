@@ -8,7 +8,7 @@ import torch
 import paper_2505_19634_b200 as tts
 import tts_inputs as ti
 
-ATTN_IMPLS = [tts.ATTN_SIMT]
+ATTN_IMPLS = [tts.ATTN_SIMT, tts.ATTN_TCGEN05]
 IMPL_NAMES = {tts.ATTN_SIMT: "simt", tts.ATTN_TCGEN05: "tcgen05", tts.ATTN_AUTO: "auto"}
 
 
