@@ -49,8 +49,12 @@ typedef enum {
 enum { TTS_MASK_CAUSAL = 0, TTS_MASK_TREE = 1 };
 enum { TTS_OUT_BF16 = 0, TTS_OUT_FP32 = 1 };
 /* Which attention kernel runs: AUTO picks tensor cores (tcgen05, TMEM accumulators) when the
- * stacked query rows per KV head make it worthwhile and CUDA cores otherwise. */
-enum { TTS_ATTN_AUTO = 0, TTS_ATTN_SIMT = 1, TTS_ATTN_TCGEN05 = 2 };
+ * stacked query rows per KV head make it worthwhile and CUDA cores otherwise.  TCGEN05 picks
+ * between the two tensor-core kernels: TOKEN_MAJOR (KV tokens on the MMA M dimension, for at most
+ * 64 rows per branch and KV head: chains of gamma+1 positions) and ROW_MAJOR (query rows on M, for
+ * draft trees with many nodes).  The last two force one of them. */
+enum { TTS_ATTN_AUTO = 0, TTS_ATTN_SIMT = 1, TTS_ATTN_TCGEN05 = 2, TTS_ATTN_TCGEN05_TOKEN_MAJOR = 3,
+       TTS_ATTN_TCGEN05_ROW_MAJOR = 4 };
 
 typedef struct tts_ctx tts_ctx;
 

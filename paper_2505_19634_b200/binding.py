@@ -16,7 +16,7 @@ _LIB_PATH = _PKG / "libtts_b200.so"
 
 MASK_CAUSAL, MASK_TREE = 0, 1
 OUT_BF16, OUT_FP32 = 0, 1
-ATTN_AUTO, ATTN_SIMT, ATTN_TCGEN05 = 0, 1, 2
+ATTN_AUTO, ATTN_SIMT, ATTN_TCGEN05, ATTN_TCGEN05_TOKEN_MAJOR, ATTN_TCGEN05_ROW_MAJOR = 0, 1, 2, 3, 4
 
 EXPORTED_SYMBOLS = (
     "tts_create", "tts_destroy", "tts_set_stream", "tts_verify_attn", "tts_verify_attn_tree",

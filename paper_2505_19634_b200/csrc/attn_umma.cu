@@ -31,10 +31,13 @@
 #include <vector>
 
 #include "tts_internal.cuh"
+#include "umma_ptx.cuh"
 
 namespace tts {
 
 namespace {
+
+using namespace ptx;
 
 constexpr int kTile = kUmmaTileTokens;            // 128 tokens
 constexpr int kRows = kUmmaRows;                   // 128 = MMA M
@@ -43,7 +46,6 @@ constexpr int kHalfBytes = kRows * 128;            // one 64-element K-block of 
 constexpr int kOperandBytes = 2 * kHalfBytes;      // 32 KiB
 constexpr int kRing = 2;
 constexpr uint32_t kTmemCols = 512;
-constexpr long long kWaitLimitNs = 400ll * 1000 * 1000;
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int kOffQ = 0;
@@ -59,125 +61,8 @@ constexpr int kSmemBytes = kOffCum + (kUmmaMaxBranches + 1) * 4 + 1024;   // + s
 
 enum Bar { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, S_FULL = 8, S_FREE = 10, P_FULL = 12, PV_DONE = 13, Q_FULL = 14 };
 
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ long long global_ns() {
-    long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-struct Abort {
-    volatile int* flag;     // shared: set when any wait of this CTA ran out
-    int32_t* status;        // global status word
-};
-
-// Bounded wait.  Returns false if the CTA is aborting (this or another wait ran out of time).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = global_ns();
-    for (int spin = 0;; ++spin) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 63) == 63) {
-            if (*ab.flag) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
-                *ab.flag = 1;
-                atomicMin(ab.status, (int)TTS_ERR_DEVICE_TIMEOUT);
-                return false;
-            }
-        }
-    }
-}
-
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
-          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-        : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ float ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-// Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).
-//   K-major operand  (rows x 64-element K-block, 128-byte rows): lbo = 16, sbo = 1024 (8-row atoms)
-//   MN-major operand (64-element MN-block x K rows):             lbo = bytes between MN-blocks,
-//                                                                 sbo = 1024 (8 K-rows)
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)(lbo_bytes >> 4) << 16;
-    d |= (uint64_t)(sbo_bytes >> 4) << 32;
-    d |= 1ull << 46;                      // descriptor version
-    d |= 2ull << 61;                      // SWIZZLE_128B
-    return d;
-}
-
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128; B either K-major or MN-major.
-__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-}
-
+__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) { return ptx::instr_desc(128, 128, false, b_mn_major); }
 // byte offset of the 16-byte chunk holding elements [8*chunk, 8*chunk+8) of `row` in a 128-row,
 // 128-element-wide K-major operand with 128-byte swizzle
 __device__ __forceinline__ uint32_t kmajor_chunk_off(int row, int chunk) {
@@ -550,8 +435,10 @@ EncodeTiledFn encode_fn() {
 struct MapEntry { const void* ptr; long rows; CUtensorMap map; };
 struct MapCache { std::vector<MapEntry> entries; };
 
+}  // namespace
+
 // 2-D view of a page pool: rows = num_pages * Hkv * 16 tokens of 128 bf16; box = 64 dims x 16 tokens.
-const CUtensorMap* pool_map(Ctx* c, const void* pool, cudaError_t* err) {
+const CUtensorMap* umma_pool_map(Ctx* c, const void* pool, cudaError_t* err) {
     if (!c->tmap_cache) c->tmap_cache = new MapCache();
     MapCache* mc = static_cast<MapCache*>(c->tmap_cache);
     const long rows = (long)c->cfg.num_pages * c->cfg.n_kv_heads * kPage;
@@ -574,8 +461,6 @@ const CUtensorMap* pool_map(Ctx* c, const void* pool, cudaError_t* err) {
     return &mc->entries.back().map;
 }
 
-}  // namespace
-
 bool umma_available() { return true; }
 
 int umma_copies(int nr) { return nr <= 32 ? 4 : (nr <= 64 ? 2 : 1); }
@@ -583,10 +468,10 @@ int umma_copies(int nr) { return nr <= 32 ? 4 : (nr <= 64 ? 2 : 1); }
 cudaError_t launch_attn_umma(Ctx* c, const AttnParams& p, cudaStream_t st) {
     if (p.N > kUmmaMaxBranches) return cudaErrorInvalidValue;
     cudaError_t err = cudaSuccess;
-    const CUtensorMap* mk = pool_map(c, p.k_pages, &err);
+    const CUtensorMap* mk = umma_pool_map(c, p.k_pages, &err);
     if (!mk) return err;
     const CUtensorMap mk_copy = *mk;                       // the cache may reallocate on the next insert
-    const CUtensorMap* mv = pool_map(c, p.v_pages, &err);
+    const CUtensorMap* mv = umma_pool_map(c, p.v_pages, &err);
     if (!mv) return err;
     static bool attr_set[64] = {};                          // the attribute is per device
     if (c->device < 0 || c->device >= 64 || !attr_set[c->device]) {

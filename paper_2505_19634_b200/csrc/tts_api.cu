@@ -25,8 +25,12 @@ Plan make_plan(const Ctx* c, int nr) {
     Plan pl;
     int impl = c->cfg.attn_impl;
     if (impl == TTS_ATTN_AUTO) impl = umma_available() && nr >= kUmmaMinRows ? TTS_ATTN_TCGEN05 : TTS_ATTN_SIMT;
+    // few rows per KV head: KV tokens on the MMA M dimension; many (draft trees): query rows on M
+    if (impl == TTS_ATTN_TCGEN05) impl = nr <= kUmmaTMaxRows ? TTS_ATTN_TCGEN05_TOKEN_MAJOR : TTS_ATTN_TCGEN05_ROW_MAJOR;
     pl.impl = impl;
-    if (impl == TTS_ATTN_TCGEN05) {
+    if (impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR) {
+        pl.rb_rows = umma_t_rows(nr); pl.tile_tokens = kUmmaTileTokens; pl.grid = c->n_sms; pl.copies = 1;
+    } else if (impl == TTS_ATTN_TCGEN05_ROW_MAJOR) {
         pl.rb_rows = kUmmaRows; pl.tile_tokens = kUmmaTileTokens; pl.grid = c->n_sms;
         pl.copies = nr <= kUmmaRows ? umma_copies(nr) : 1;
     } else {
@@ -58,10 +62,10 @@ cudaError_t alloc_workspace(Ctx* c) {
     const int G = f.n_q_heads / f.n_kv_heads;
     const int nr = f.max_rows_per_branch * G;
     size_t pre = 0, priv = 0;
-    const int cand_rb[4] = {8, 16, 32, kUmmaRows};
-    for (int k = 0; k < 4; ++k) {
+    const int cand_rb[5] = {8, 16, 32, 64, kUmmaRows};
+    for (int k = 0; k < 5; ++k) {
         // a call may carry fewer rows than the maximum and then replicate them more often
-        for (int copies = 1; copies <= (k == 3 ? 4 : 1); copies *= 2) {
+        for (int copies = 1; copies <= (k == 4 ? 4 : 1); copies *= 2) {
             const int nr_c = copies == 1 ? nr : (nr < kUmmaRows / copies ? nr : kUmmaRows / copies);
             size_t a, b;
             workspace_rows(f.max_branches, f.n_kv_heads, nr_c, cand_rb[k], copies, c->n_sms * 3, &a, &b);
@@ -132,7 +136,9 @@ int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
     const bool prof = c->profiling && c->prof_ev && c->prof_n < kProfMaxCalls;
     cudaEvent_t* ev = prof ? c->prof_ev + 3 * c->prof_n : nullptr;
     if (prof) cudaEventRecord(ev[0], c->stream);
-    if (pl.impl == TTS_ATTN_TCGEN05) {
+    if (pl.impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR) {
+        e = launch_attn_umma_t(c, p, c->stream);
+    } else if (pl.impl == TTS_ATTN_TCGEN05_ROW_MAJOR) {
         if (!umma_available()) return TTS_ERR_UNSUPPORTED;
         e = launch_attn_umma(c, p, c->stream);
     } else {
@@ -161,7 +167,7 @@ int tts_create(const tts_config* cfg, tts_ctx** out) {
     if (cfg->max_rows_per_branch < 1 || cfg->max_rows_per_branch > kMaxTreeRows) return TTS_ERR_INVALID;
     if (cfg->max_blocks_per_branch < 1 || cfg->num_pages < 1) return TTS_ERR_INVALID;
     if (cfg->out_dtype != TTS_OUT_BF16 && cfg->out_dtype != TTS_OUT_FP32) return TTS_ERR_UNSUPPORTED;
-    if (cfg->attn_impl < TTS_ATTN_AUTO || cfg->attn_impl > TTS_ATTN_TCGEN05) return TTS_ERR_UNSUPPORTED;
+    if (cfg->attn_impl < TTS_ATTN_AUTO || cfg->attn_impl > TTS_ATTN_TCGEN05_ROW_MAJOR) return TTS_ERR_UNSUPPORTED;
     if (!(cfg->softmax_scale >= 0.f)) return TTS_ERR_INVALID;
 
     Ctx* c = new (std::nothrow) Ctx();

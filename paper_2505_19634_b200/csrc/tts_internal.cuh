@@ -190,6 +190,10 @@ constexpr int kUmmaMinRows = 9;        // below this many stacked rows per KV he
 bool umma_available();
 int umma_copies(int nr);              // replication factor of a private piece's rows along the MMA M dimension
 cudaError_t launch_attn_umma(Ctx* c, const AttnParams& p, cudaStream_t st);
+// token-major tcgen05 kernel (KV tokens on the MMA M dimension): row blocks of 32 or 64 stacked rows
+constexpr int kUmmaTMaxRows = 64;
+int umma_t_rows(int nr);
+cudaError_t launch_attn_umma_t(Ctx* c, const AttnParams& p, cudaStream_t st);
 void umma_release(Ctx* c);
 
 }  // namespace tts

@@ -8,8 +8,9 @@ import torch
 import paper_2505_19634_b200 as tts
 import tts_inputs as ti
 
-ATTN_IMPLS = [tts.ATTN_SIMT, tts.ATTN_TCGEN05]
-IMPL_NAMES = {tts.ATTN_SIMT: "simt", tts.ATTN_TCGEN05: "tcgen05", tts.ATTN_AUTO: "auto"}
+ATTN_IMPLS = [tts.ATTN_SIMT, tts.ATTN_TCGEN05_TOKEN_MAJOR, tts.ATTN_TCGEN05_ROW_MAJOR]
+IMPL_NAMES = {tts.ATTN_SIMT: "simt", tts.ATTN_TCGEN05: "tcgen05", tts.ATTN_AUTO: "auto",
+              tts.ATTN_TCGEN05_TOKEN_MAJOR: "tcgen05_token_major", tts.ATTN_TCGEN05_ROW_MAJOR: "tcgen05_row_major"}
 
 
 def dev_bf16(bits: np.ndarray) -> torch.Tensor:
