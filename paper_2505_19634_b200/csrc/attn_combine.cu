@@ -10,29 +10,15 @@ namespace {
 constexpr int kRowsPerBlock = 4;
 
 __global__ void __launch_bounds__(kRowsPerBlock * 32) attn_combine_kernel(const AttnParams p) {
+    extern __shared__ int cum[];                                         // N + 1 ints
+    build_branch_tile_prefix(p, cum);
     const int lane = threadIdx.x & 31;
     const int row = blockIdx.x * kRowsPerBlock + (threadIdx.x >> 5);     // (b, i, h) flattened
     if (row >= p.N * p.R * p.Hq) return;
     const int h = row % p.Hq, i = (row / p.Hq) % p.R, b = row / (p.Hq * p.R);
     const int kvh = h / p.G, gq = h % p.G;
-
-    // tiles of the branches before b, of b, and of all branches (lanes stride over branches)
-    int before = 0, all = 0;
-    for (int bb = lane; bb < p.N; bb += 32) {
-        int L = p.branch_lens[bb];
-        const int t = ceil_div(L < 0 ? 0 : L, p.tile_tokens);
-        all += t;
-        if (bb < b) before += t;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        before += __shfl_xor_sync(0xffffffffu, before, o);
-        all += __shfl_xor_sync(0xffffffffu, all, o);
-    }
-    const int tiles_b = ceil_div(max(p.branch_lens[b], 0), p.tile_tokens);
-    const int per = p.Hkv * p.n_rb_priv;
-    const int pre_total = p.n_pre * p.tiles_pre;
-    const int total = pre_total + per * all;
+    const int tiles_b = cum[b + 1] - cum[b];
+    const int total = total_tiles(p, cum);
     const int tpc = ceil_div(total, p.grid);
 
     float m_run = -INFINITY, l_run = 0.f;
@@ -66,14 +52,13 @@ __global__ void __launch_bounds__(kRowsPerBlock * 32) attn_combine_kernel(const 
         const int pr = b * p.nr + r_priv;
         const int rb = pr / p.rb_rows, r = pr % p.rb_rows;
         const int seg = kvh * p.n_rb_pre + rb;
-        merge(p.part_o_pre, p.part_ml_pre, p.pre_stride, seg, r, 0, 1, seg * p.tiles_pre, p.tiles_pre);
+        merge(p.part_o_pre, p.part_ml_pre, p.pre_stride, seg, r, 0, 1, prefix_segment_tile_begin(p, cum, seg), p.tiles_pre);
     }
     {
         const int rb = r_priv / p.rb_rows, r = r_priv % p.rb_rows;
-        const int within = kvh * p.n_rb_priv + rb;
-        const int seg = b * per + within;
+        const int seg = (b * p.Hkv + kvh) * p.n_rb_priv + rb;
         merge(p.part_o_priv, p.part_ml_priv, p.priv_stride, seg, r, min(p.rb_rows, p.nr - rb * p.rb_rows), p.copies,
-              pre_total + per * before + within * tiles_b, tiles_b);
+              group_tile_begin(p, cum, b * p.Hkv + kvh) + rb * tiles_b, tiles_b);
     }
 
     const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
@@ -93,7 +78,7 @@ __global__ void __launch_bounds__(kRowsPerBlock * 32) attn_combine_kernel(const 
 
 cudaError_t launch_attn_combine(const AttnParams& p, cudaStream_t st) {
     const int rows = p.N * p.R * p.Hq;
-    attn_combine_kernel<<<ceil_div(rows, kRowsPerBlock), kRowsPerBlock * 32, 0, st>>>(p);
+    attn_combine_kernel<<<ceil_div(rows, kRowsPerBlock), kRowsPerBlock * 32, (p.N + 1) * sizeof(int), st>>>(p);
     return cudaGetLastError();
 }
 

@@ -264,6 +264,9 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                     uint4 v = make_uint4(0, 0, 0, 0);
                     if (valid) v = __ldg(reinterpret_cast<const uint4*>(src) + c);
                     *reinterpret_cast<uint4*>(smem + kOffQ + kmajor_chunk_off(L, c)) = v;
+                    // a copy only ever writes its own column slice of its P row: the rest must be zero
+                    // (the previous piece's last P.V has completed, see the piece epilogue)
+                    if (ncopy > 1) *reinterpret_cast<uint4*>(smem + kOffP + kmajor_chunk_off(L, c)) = make_uint4(0, 0, 0, 0);
                 }
             }
             fence_proxy_async();

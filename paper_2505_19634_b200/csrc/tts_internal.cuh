@@ -19,13 +19,17 @@ constexpr int kMaxBranches = 1024;
 //   prefix segments   s = kvh * n_rb_pre + rb            rows = all branches' rows, stacked
 //                                                          (b, i, g) -> b*nr + i*G + g; every row
 //                                                          sees every prefix token (no mask)
-//   private segments  s = n_pre + (b*Hkv + kvh) * n_rb_priv + rb   rows = (i, g) -> i*G + g
+//   private segments  (b, kvh, rb)                         rows = (i, g) -> i*G + g
 // Each segment is cut into tiles of tile_tokens KV tokens; all tiles of all segments form one
 // global list, and CTA c of a persistent grid owns the contiguous run [c*tpc, (c+1)*tpc) of it
-// (tpc = ceil(total / grid)).  The run of one CTA inside one segment is a *piece*; it produces
-// one partial result (running max m, sum l, unnormalised O) per row.  Because segments and CTAs
-// advance together along the list, (segment + CTA) is a unique index for every piece, so no
-// scan over pieces is needed to place them in the workspace.
+// (tpc = ceil(total / grid)).  The list goes group by group, a group being the n_rb_priv private
+// segments of one (branch, KV head), idx = b*Hkv + kvh; the prefix segments are spread evenly
+// between the groups (segments [pre_before(idx), pre_before(idx+1)) follow group idx), so that no
+// CTA gets more than a few of these short segments.  The run of one CTA inside one segment is a
+// *piece*; it produces one partial result (running max m, sum l, unnormalised O) per row.  Because
+// segments of either kind and CTAs both advance along the list, (segment index within its kind +
+// CTA) is a unique index for every piece, so no scan over pieces is needed to place them in the
+// workspace.
 struct AttnParams {
     const __nv_bfloat16* q;
     const __nv_bfloat16* k_pages;
@@ -70,54 +74,90 @@ __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; 
 // cum[b] = tiles of branches < b (per private segment of that branch), cum[N] = sum.
 // Must be called by all threads of the block; cum lives in shared memory (N+1 ints).
 __device__ inline void build_branch_tile_prefix(const AttnParams& p, int* cum) {
-    if (threadIdx.x == 0) {
-        int run = 0;
-        for (int b = 0; b < p.N; ++b) {
-            cum[b] = run;
-            int L = p.branch_lens[b];
-            L = L < 0 ? 0 : L;
-            run += ceil_div(L, p.tile_tokens);
+    for (int b = threadIdx.x; b < p.N; b += blockDim.x) {
+        int L = p.branch_lens[b];
+        L = L < 0 ? 0 : L;
+        cum[b + 1] = ceil_div(L, p.tile_tokens);
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {                                  // inclusive scan by the first warp, 32 at a time
+        const int lane = threadIdx.x;
+        int carry = 0;
+        for (int base = 0; base < p.N; base += 32) {
+            int v = base + lane < p.N ? cum[base + lane + 1] : 0;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int n = __shfl_up_sync(0xffffffffu, v, o);
+                if (lane >= o) v += n;
+            }
+            if (base + lane < p.N) cum[base + lane + 1] = carry + v;
+            carry += __shfl_sync(0xffffffffu, v, 31);
         }
-        cum[p.N] = run;
+        if (lane == 0) cum[0] = 0;
     }
     __syncthreads();
 }
 
+// prefix segments placed before group idx (idx in [0, N*Hkv])
+__device__ inline int pre_before(const AttnParams& p, int idx) {
+    return (int)((long long)idx * p.n_pre / (p.N * p.Hkv));
+}
+
+// global index of the first tile of group idx (idx == N*Hkv gives the total)
+__device__ inline int group_tile_begin(const AttnParams& p, const int* cum, int idx) {
+    const int b = idx / p.Hkv, kvh = idx - b * p.Hkv;
+    const int tb = b < p.N ? cum[b + 1] - cum[b] : 0;
+    return p.n_rb_priv * (p.Hkv * cum[b] + kvh * tb) + p.tiles_pre * pre_before(p, idx);
+}
+
 __device__ inline int total_tiles(const AttnParams& p, const int* cum) {
-    return p.n_pre * p.tiles_pre + p.Hkv * p.n_rb_priv * cum[p.N];
+    return group_tile_begin(p, cum, p.N * p.Hkv);
+}
+
+__device__ inline SegInfo prefix_segment(const AttnParams& p, int s, int tile_begin) {
+    SegInfo g;
+    g.kind = 0; g.b = -1;
+    g.kvh = s / p.n_rb_pre; g.rb = s % p.n_rb_pre;
+    g.row0 = g.rb * p.rb_rows;
+    g.n_rows = min(p.rb_rows, p.N * p.nr - g.row0);
+    g.tile_begin = tile_begin; g.n_tiles = p.tiles_pre;
+    g.tok_begin = 0; g.n_tokens = p.P;
+    return g;
 }
 
 // Segment that contains global tile g (0 <= g < total).
 __device__ inline SegInfo segment_of_tile(const AttnParams& p, const int* cum, int g) {
-    SegInfo s;
-    const int pre_total = p.n_pre * p.tiles_pre;
-    if (g < pre_total) {
-        const int idx = g / p.tiles_pre;
-        s.kind = 0; s.b = -1;
-        s.kvh = idx / p.n_rb_pre; s.rb = idx % p.n_rb_pre;
-        s.row0 = s.rb * p.rb_rows;
-        s.n_rows = min(p.rb_rows, p.N * p.nr - s.row0);
-        s.tile_begin = idx * p.tiles_pre; s.n_tiles = p.tiles_pre;
-        s.tok_begin = 0; s.n_tokens = p.P;
-        return s;
-    }
-    const int per = p.Hkv * p.n_rb_priv;
-    const int gp = g - pre_total;
-    int lo = 0, hi = p.N - 1;                  // largest b with per*cum[b] <= gp
+    int lo = 0, hi = p.N * p.Hkv - 1;          // largest group whose first tile is <= g
     while (lo < hi) {
-        int mid = (lo + hi + 1) >> 1;
-        if (per * cum[mid] <= gp) lo = mid; else hi = mid - 1;
+        const int mid = (lo + hi + 1) >> 1;
+        if (group_tile_begin(p, cum, mid) <= g) lo = mid; else hi = mid - 1;
     }
-    const int b = lo;
+    const int idx = lo, b = idx / p.Hkv, kvh = idx - b * p.Hkv;
+    const int begin = group_tile_begin(p, cum, idx);
     const int tb = cum[b + 1] - cum[b];
-    const int within = (gp - per * cum[b]) / tb;      // (kvh, rb) index inside the branch
-    s.kind = 1; s.b = b;
-    s.kvh = within / p.n_rb_priv; s.rb = within % p.n_rb_priv;
+    const int priv_tiles = p.n_rb_priv * tb;
+    const int within = g - begin;
+    if (within >= priv_tiles) {                 // one of the prefix segments that follow the group
+        const int k = (within - priv_tiles) / p.tiles_pre;
+        return prefix_segment(p, pre_before(p, idx) + k, begin + priv_tiles + k * p.tiles_pre);
+    }
+    SegInfo s;
+    s.kind = 1; s.b = b; s.kvh = kvh;
+    s.rb = within / tb;
     s.row0 = s.rb * p.rb_rows;
     s.n_rows = min(p.rb_rows, p.nr - s.row0);
-    s.tile_begin = pre_total + per * cum[b] + within * tb; s.n_tiles = tb;
+    s.tile_begin = begin + s.rb * tb; s.n_tiles = tb;
     s.tok_begin = p.P; s.n_tokens = p.branch_lens[b];
     return s;
+}
+
+// First tile of prefix segment s: it follows the first group idx with pre_before(idx + 1) > s.
+__device__ inline int prefix_segment_tile_begin(const AttnParams& p, const int* cum, int s) {
+    const long long n_groups = (long long)p.N * p.Hkv;
+    const int idx = (int)(((long long)(s + 1) * n_groups + p.n_pre - 1) / p.n_pre) - 1;
+    const int b = idx / p.Hkv;
+    const int tb = cum[b + 1] - cum[b];
+    return group_tile_begin(p, cum, idx) + p.n_rb_priv * tb + (s - pre_before(p, idx)) * p.tiles_pre;
 }
 
 __device__ inline int segment_index(const AttnParams& p, const SegInfo& s) {
