@@ -52,7 +52,8 @@ __global__ void __launch_bounds__(kRowsPerBlock * 32) attn_combine_kernel(const 
         const int pr = b * p.nr + r_priv;
         const int rb = pr / p.rb_rows, r = pr % p.rb_rows;
         const int seg = kvh * p.n_rb_pre + rb;
-        merge(p.part_o_pre, p.part_ml_pre, p.pre_stride, seg, r, 0, 1, prefix_segment_tile_begin(p, cum, seg), p.tiles_pre);
+        merge(p.part_o_pre, p.part_ml_pre, p.pre_stride, seg, r, min(p.rb_rows, p.N * p.nr - rb * p.rb_rows), p.copies_pre,
+              prefix_segment_tile_begin(p, cum, seg), p.tiles_pre);
     }
     {
         const int rb = r_priv / p.rb_rows, r = r_priv % p.rb_rows;

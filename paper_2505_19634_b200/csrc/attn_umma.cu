@@ -435,29 +435,44 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-struct MapEntry { const void* ptr; long rows; CUtensorMap map; };
+struct MapEntry { const void* ptr; long rows; int kind; CUtensorMap map; };
 struct MapCache { std::vector<MapEntry> entries; };
 
 }  // namespace
 
-// 2-D view of a page pool: rows = num_pages * Hkv * 16 tokens of 128 bf16; box = 64 dims x 16 tokens.
-const CUtensorMap* umma_pool_map(Ctx* c, const void* pool, cudaError_t* err) {
+// Tensor maps over a page pool [num_pages][Hkv][16 tokens][128 dims] bf16, 128-byte swizzle.
+//   kind 0: 2-D view, rows = num_pages * Hkv * 16 tokens of 128 dims; box = 64 dims x 16 tokens.
+//   kind 1: 5-D view (64 dims, 8 tokens, 2 dim halves, 2 token halves, page-head); box = one whole
+//           page-head tile (4 KiB), which lands as [token half][dim half][8 tokens][128 bytes]: the
+//           8-token atoms of one dim half are then 2 KiB apart across the pages of a 128-token tile.
+const CUtensorMap* umma_pool_map(Ctx* c, const void* pool, int kind, cudaError_t* err) {
     if (!c->tmap_cache) c->tmap_cache = new MapCache();
     MapCache* mc = static_cast<MapCache*>(c->tmap_cache);
     const long rows = (long)c->cfg.num_pages * c->cfg.n_kv_heads * kPage;
     for (auto& e : mc->entries)
-        if (e.ptr == pool && e.rows == rows) return &e.map;
+        if (e.ptr == pool && e.rows == rows && e.kind == kind) return &e.map;
     EncodeTiledFn fn = encode_fn();
     if (!fn) { *err = cudaErrorNotSupported; return nullptr; }
     MapEntry e;
-    e.ptr = pool; e.rows = rows;
-    const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)kPage};
-    const cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(pool), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    e.ptr = pool; e.rows = rows; e.kind = kind;
+    CUresult r;
+    if (kind == 0) {
+        const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
+        const cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
+        const cuuint32_t box[2] = {64, (cuuint32_t)kPage};
+        const cuuint32_t estr[2] = {1, 1};
+        r = fn(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(pool), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        const cuuint64_t dims[5] = {64, 8, 2, 2, (cuuint64_t)(rows / kPage)};
+        const cuuint64_t strides[4] = {256, 128, 2048, 4096};          // bytes, dimensions 1..4
+        const cuuint32_t box[5] = {64, 8, 2, 2, 1};
+        const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+        r = fn(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(pool), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
     if (r != CUDA_SUCCESS) { *err = cudaErrorInvalidValue; return nullptr; }
     if (mc->entries.size() >= 512) mc->entries.erase(mc->entries.begin());
     mc->entries.push_back(e);
@@ -471,10 +486,10 @@ int umma_copies(int nr) { return nr <= 32 ? 4 : (nr <= 64 ? 2 : 1); }
 cudaError_t launch_attn_umma(Ctx* c, const AttnParams& p, cudaStream_t st) {
     if (p.N > kUmmaMaxBranches) return cudaErrorInvalidValue;
     cudaError_t err = cudaSuccess;
-    const CUtensorMap* mk = umma_pool_map(c, p.k_pages, &err);
+    const CUtensorMap* mk = umma_pool_map(c, p.k_pages, 0, &err);
     if (!mk) return err;
     const CUtensorMap mk_copy = *mk;                       // the cache may reallocate on the next insert
-    const CUtensorMap* mv = umma_pool_map(c, p.v_pages, &err);
+    const CUtensorMap* mv = umma_pool_map(c, p.v_pages, 0, &err);
     if (!mv) return err;
     static bool attr_set[64] = {};                          // the attribute is per device
     if (c->device < 0 || c->device >= 64 || !attr_set[c->device]) {

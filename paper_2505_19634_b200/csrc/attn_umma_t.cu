@@ -9,19 +9,28 @@
 // small (NB x 256 bytes), which leaves room for a ring of 5-6 operand tiles (32 KiB each) in shared
 // memory, the depth that hides HBM latency at 4 KiB page granularity.
 //
-// One persistent CTA per SM walks its run of the global tile list (tts_internal.cuh):
-//   warp 4*CG   producer: per tile arms the "full" barrier of the next ring slot with the byte count
-//               and issues the TMA boxes of the K tile, then of the V tile (8 pages x 2 boxes each)
-//   warp 4*CG+1 MMA issuer (one thread): S^T into one of two TMEM buffers, O^T (+)= V^T P^T once the
-//               softmax warps have published P^T; tcgen05.commit frees ring slots and P buffers
-//   warps 0..4*CG-1  softmax: thread = (TMEM lane = KV token, column group).  The NB rows are cut
-//               into chunks of 4; column group cg owns chunks cg, cg+CG, ... and a thread holds the
-//               scores of its token for the rows of its chunks (chunks past the piece's last row are
-//               skipped).  The running reference m of every row lives in shared memory and only
-//               moves when some score exceeds it by more than 2^8 (consensus through a reducing
-//               named barrier; the exact row maximum is then found with warp redux + shared memory
-//               and O^T is rescaled in TMEM).  The result is exact either way: l is accumulated
-//               against the same reference.  Row sums are kept per thread and reduced once per piece.
+// One persistent CTA per SM walks its run of the global tile list (tts_internal.cuh), two tiles
+// (256 tokens) per step: the latency chain of a step (MMA -> TMEM load -> consensus -> exp -> P^T
+// -> MMA) is paid once for both tiles, and every thread works on two independent tokens.
+//
+//   producer warp    per step arms the "full" barriers of the next ring slots with the byte counts and
+//                    issues the TMA copies of the K tiles, then of the V tiles: one 5-D box per page-head
+//                    tile (4 KiB), laid out so that the 8 pages of a tile form one MMA operand
+//   MMA warp         one thread: S^T of the step's tiles into one of two pairs of TMEM buffers (the
+//                    next step's scores are computed while the softmax warps work on this one's),
+//                    O^T (+)= V^T P^T once P^T has been published; tcgen05.commit frees ring slots,
+//                    P buffers and, at the end of a piece, the Q block
+//   softmax warps    4*CG warps: thread = (TMEM lane = KV token of either tile, column group).  The NB
+//                    rows are cut into chunks of 4; column group cg owns chunks cg, cg+CG, ... and a
+//                    thread holds the scores of its tokens for the rows of its chunks (chunks past the
+//                    piece's last row are skipped).  The running reference m of every row lives in
+//                    shared memory and only moves when some score exceeds it by more than 2^8
+//                    (consensus through a reducing named barrier; the exact row maximum is then found
+//                    with warp redux + shared memory and O^T is rescaled in TMEM).  The result is
+//                    exact either way: l is accumulated against the same reference.  Row sums are kept
+//                    per thread and reduced once per piece.  The Q block of the next piece is
+//                    prefetched into registers and stored once the MMA issuer has signalled that the
+//                    current piece no longer reads Q.
 //
 // Every wait is bounded.  A wait that runs out raises TTS_ERR_DEVICE_TIMEOUT; the softmax warps only
 // leave their loops on the result of a block-wide reduction, so no thread is left behind at a named
@@ -39,7 +48,6 @@ using namespace ptx;
 
 constexpr int kTileT = kUmmaTileTokens;              // 128 tokens = MMA M
 constexpr int kSlotBytes = kTileT * kHeadDim * 2;    // one K or V tile: 32 KiB
-constexpr int kHalfT = kTileT * 128;                 // one 64-element block of a 128-row operand: 16 KiB
 constexpr float kLazy = 8.f;                         // the reference moves when exceeded by 2^8
 
 template <int NB>
@@ -48,35 +56,42 @@ struct Lay {
     static constexpr int kQBytes = NB * 256;         // two 64-dim K-blocks of NB rows x 128 B
     static constexpr int kPBytes = NB * 256;         // two 64-token K-blocks of NB rows x 128 B
     static constexpr int kOffQ = 0;
-    static constexpr int kOffP = kQBytes;            // two buffers
+    static constexpr int kOffP = kQBytes;            // one buffer per tile of a step
     static constexpr int kOffRing = kOffP + 2 * kPBytes;
     static constexpr int kOffBar = kOffRing + kSlots * kSlotBytes;
-    static constexpr int kOffMisc = kOffBar + 24 * 8;            // 2 * kSlots + 9 barriers
+    static constexpr int kOffMisc = kOffBar + 24 * 8;            // 2 * kSlots + 8 barriers
     static constexpr int kOffMref = kOffMisc + 64;               // float[NB]
     static constexpr int kOffRed = kOffMref + NB * 4;            // float[4][NB]
     static constexpr int kOffVis = kOffRed + 4 * NB * 4;         // u64[64]
     static constexpr int kOffCum = kOffVis + 64 * 8;             // int[N + 1]
     static constexpr int kFixedBytes = kOffCum + 1024;           // + slack for the manual 1024-B alignment
-    static constexpr uint32_t kTmemCols = NB == 32 ? 128 : 256;  // 2 S^T buffers + O^T, power of two
+    static constexpr uint32_t kTmemCols = NB == 32 ? 256 : 512;  // 2 pairs of S^T buffers + O^T, power of two
     // barrier indices
     static constexpr int FULL = 0, EMPTY = kSlots, S_FULL = 2 * kSlots, S_FREE = S_FULL + 2, P_FULL = S_FREE + 2,
-                         P_FREE = P_FULL + 2, Q_FULL = P_FREE + 2;
+                         P_FREE = P_FULL + 1, Q_FULL = P_FREE + 1, Q_FREE = Q_FULL + 1;
 };
 
-// reducing / plain named barrier 1 over the NT softmax threads
+// reducing / plain named barrier `id` over NT threads
 template <int NT>
-__device__ __forceinline__ bool bar_red_or(bool pred) {
+__device__ __forceinline__ bool bar_red_or(int id, bool pred) {
     uint32_t out;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.u32 q, %1, 0;\n\t"
-        "barrier.cta.red.or.pred p, 1, %2, q;\n\t"
+        "barrier.cta.red.or.pred p, %2, %3, q;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(out) : "r"((uint32_t)pred), "n"(NT) : "memory");
+        : "=r"(out) : "r"((uint32_t)pred), "r"(id), "n"(NT) : "memory");
     return out != 0;
 }
 template <int NT>
-__device__ __forceinline__ void bar_sync_softmax() { asm volatile("barrier.cta.sync 1, %0;" ::"n"(NT) : "memory"); }
+__device__ __forceinline__ void bar_sync_id(int id) { asm volatile("barrier.cta.sync %0, %1;" ::"r"(id), "n"(NT) : "memory"); }
+
+// One mbarrier arrival for the whole warp, after every lane's preceding work (arrivals of single
+// threads on one barrier serialise, so the barriers count warps).
+__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+}
 
 __device__ __forceinline__ float warp_max_f32(float v) {
     int i = __float_as_int(v);
@@ -102,25 +117,42 @@ __device__ __forceinline__ void tmem_st4(uint32_t taddr, const float* v) {
                  ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
 }
 
-// Q block of a piece -> shared memory as the K-major B operand (zero rows beyond n_rows), and, for
-// private segments under a tree mask, the visibility word of every query position.
+// The Q block of a piece, fetched by the NT threads of group 0 (QPT 16-byte chunks each) and later
+// stored as the K-major B operand (zero rows beyond n_rows).
 template <int NB, int NT>
-__device__ __forceinline__ void stage_q(const AttnParams& p, const SegInfo& seg, unsigned char* smem, int tid) {
-    using L = Lay<NB>;
-    for (int idx = tid; idx < NB * 16; idx += NT) {
-        const int r = idx >> 4, c = idx & 15;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (r < seg.n_rows) {
-            int row = seg.row0 + r, b = seg.b;
-            if (seg.kind == 0) { b = row / p.nr; row = row % p.nr; }
-            const int i = row / p.G, gq = row % p.G;
-            const __nv_bfloat16* src = p.q + (((size_t)b * p.R + i) * p.Hq + seg.kvh * p.G + gq) * kHeadDim;
-            v = __ldg(reinterpret_cast<const uint4*>(src) + c);
+struct QFetch {
+    static constexpr int QPT = NB * 16 / NT;
+    uint4 v[QPT];
+    __device__ __forceinline__ void load(const AttnParams& p, const SegInfo& seg, int t) {
+#pragma unroll
+        for (int k = 0; k < QPT; ++k) {
+            const int idx = t + k * NT, r = idx >> 4, c = idx & 15;
+            v[k] = make_uint4(0, 0, 0, 0);
+            if (r < seg.n_rows) {
+                int row = seg.row0 + r, b = seg.b;
+                if (seg.kind == 0) { b = row / p.nr; row = row % p.nr; }
+                const int i = row / p.G, gq = row % p.G;
+                const __nv_bfloat16* src = p.q + (((size_t)b * p.R + i) * p.Hq + seg.kvh * p.G + gq) * kHeadDim;
+                v[k] = __ldg(reinterpret_cast<const uint4*>(src) + c);
+            }
         }
-        *reinterpret_cast<uint4*>(smem + L::kOffQ + (c >> 3) * (NB * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v;
     }
-    if (seg.kind == 1 && p.tree_parents != nullptr && tid < p.R)
-        reinterpret_cast<unsigned long long*>(smem + L::kOffVis)[tid] = row_visibility(p, seg.b, tid);
+    __device__ __forceinline__ void store(unsigned char* q_smem, int t) const {
+#pragma unroll
+        for (int k = 0; k < QPT; ++k) {
+            const int idx = t + k * NT, r = idx >> 4, c = idx & 15;
+            *reinterpret_cast<uint4*>(q_smem + (c >> 3) * (NB * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v[k];
+        }
+    }
+};
+
+// Byte offset of token `row` (dim half 0) inside a staged K or V tile: pages of 4 KiB, each
+// [token half][dim half][8 tokens][128 bytes].
+__device__ __forceinline__ int tile_row_off(int row) { return (row >> 4) * 4096 + ((row >> 3) & 1) * 2048 + (row & 7) * 128; }
+
+// Tiles of step `ss` of a piece whose tiles are [t_first, t_last): 1 or 2.
+__device__ __forceinline__ int step_tiles(int t_first, int t_last, int ss_local) {
+    return min(2, t_last - t_first - 2 * ss_local);
 }
 
 template <int NB, int CG>
@@ -130,7 +162,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     constexpr int NS = L::kSlots;
     constexpr int NT = 128 * CG;                           // softmax threads
     constexpr int NCK = NB / 4 / CG;                       // 4-row chunks per thread
-    constexpr int kProducerWarp = 4 * CG, kMmaWarp = 4 * CG + 1;
+    constexpr int kProducerWarp = 4 * CG, kMmaWarp = kProducerWarp + 1;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -151,11 +183,9 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     if (tid == 0) {
         misc[0] = 0;
         for (int i = 0; i < NS; ++i) { mbar_init(bar(L::FULL + i), 1); mbar_init(bar(L::EMPTY + i), 1); }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(bar(L::S_FULL + i), 1); mbar_init(bar(L::S_FREE + i), NT);
-            mbar_init(bar(L::P_FULL + i), NT); mbar_init(bar(L::P_FREE + i), 1);
-        }
-        mbar_init(bar(L::Q_FULL), NT);
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(L::S_FULL + i), 1); mbar_init(bar(L::S_FREE + i), 4 * CG); }
+        mbar_init(bar(L::P_FULL), 4 * CG); mbar_init(bar(L::P_FREE), 1);     // softmax warps arrive once per warp
+        mbar_init(bar(L::Q_FULL), 4 * CG); mbar_init(bar(L::Q_FREE), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMmaWarp) {
@@ -167,47 +197,51 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = (uint32_t)misc[1];
-    const uint32_t tmem_s[2] = {tmem, tmem + (uint32_t)NB};
-    const uint32_t tmem_o = tmem + 2u * NB;
+    // S^T of tile i of step ss at columns [(2 (ss & 1) + i) NB, +NB); O^T at [4 NB, +NB)
+    const uint32_t tmem_o = tmem + 4u * NB;
+    const SegInfo seg0 = segment_of_tile(p, cum, g_begin);
 
     if (warp == kProducerWarp) {
         // =========================== producer ===========================
-        int u = 0;                                          // operand tiles issued by this CTA (K, V, K, V, ...)
-        int g = g_begin;
+        int u = 0;                                          // operand tiles issued by this CTA
         bool alive = true;
-        while (g < g_end && alive) {
-            const SegInfo seg = segment_of_tile(p, cum, g);
+        SegInfo seg = seg0;
+        for (int g = g_begin;;) {
             const int t_first = g - seg.tile_begin, t_last = min(seg.n_tiles, g_end - seg.tile_begin);
             const int32_t* bt = p.block_table + (size_t)(seg.kind == 0 ? 0 : seg.b) * p.max_blocks;
-            for (int t = t_first; t < t_last && alive; ++t) {
-                const int tok0 = t * kTileT;
-                const int n_pages = ceil_div(min(kTileT, seg.n_tokens - tok0), kPage);
-                int page = 0;
-                if (lane < n_pages) {
-                    page = bt[(seg.tok_begin + tok0) / kPage + lane];
-                    if (p.debug && (page < 0 || page >= p.num_pages)) {
-                        atomicMin(p.status, (int)TTS_ERR_DEVICE_BOUNDS);
-                        page = 0;
+            for (int t = t_first; t < t_last && alive; t += 2) {
+                const int nt = min(2, t_last - t);
+                int n_pages[2] = {0, 0}, y[2] = {0, 0};
+                for (int i = 0; i < nt; ++i) {
+                    const int tok0 = (t + i) * kTileT;
+                    n_pages[i] = ceil_div(min(kTileT, seg.n_tokens - tok0), kPage);
+                    int page = 0;
+                    if (lane < n_pages[i]) {
+                        page = bt[(seg.tok_begin + tok0) / kPage + lane];
+                        if (p.debug && (page < 0 || page >= p.num_pages)) {
+                            atomicMin(p.status, (int)TTS_ERR_DEVICE_BOUNDS);
+                            page = 0;
+                        }
                     }
+                    y[i] = page * p.Hkv + seg.kvh;             // page-head index
                 }
-                const int y = (page * p.Hkv + seg.kvh) * kPage;
-#pragma unroll
-                for (int op = 0; op < 2 && alive; ++op, ++u) {
+                // ring order of a step: K tiles, then V tiles (the order the MMA issuer consumes them in)
+                for (int k = 0; k < 2 * nt && alive; ++k, ++u) {
+                    const int op = k / nt, i = k - op * nt;
                     const int slot = u % NS;
                     if (lane == 0) {
                         alive = mbar_wait(bar(L::EMPTY + slot), ((u / NS) & 1) ^ 1, ab);
-                        if (alive) mbar_arrive_expect_tx(bar(L::FULL + slot), (uint32_t)n_pages * 4096u);
+                        if (alive) mbar_arrive_expect_tx(bar(L::FULL + slot), (uint32_t)n_pages[i] * 4096u);
                     }
                     alive = __shfl_sync(0xffffffffu, alive, 0);
-                    if (alive && lane < n_pages) {
-                        const uint32_t dst = sbase + L::kOffRing + slot * kSlotBytes + lane * 2048;
-                        const CUtensorMap* tm = op == 0 ? &tm_k : &tm_v;
-                        tma_load_2d(dst, tm, 0, y, bar(L::FULL + slot));
-                        tma_load_2d(dst + kHalfT, tm, 64, y, bar(L::FULL + slot));
-                    }
+                    if (alive && lane < n_pages[i])
+                        tma_load_page(sbase + L::kOffRing + slot * kSlotBytes + lane * 4096, op == 0 ? &tm_k : &tm_v, y[i],
+                                      bar(L::FULL + slot));
                 }
             }
             g = seg.tile_begin + t_last;
+            if (g >= g_end || !alive) break;
+            seg = next_segment(p, cum, seg);
         }
         // Copies this warp started must have landed before the CTA may exit: the consumers wait on
         // the same phases in the normal case; after an abort wait for them here (bounded).
@@ -224,48 +258,65 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         if (lane == 0) {
             constexpr uint32_t idesc_qk = instr_desc(kTileT, NB, false, false);
             constexpr uint32_t idesc_pv = instr_desc(kTileT, NB, true, false);
-            int it = 0, piece = 0;
-            int g = g_begin;
+            int ss = 0, piece = 0;                           // steps / pieces of this CTA so far
+            int u_qk = 0;                                    // ring position of the next step's first K tile
             bool alive = true;
-            auto issue_qk = [&](int j) -> bool {
-                const int u = 2 * j, slot = u % NS, sb = j & 1;
-                if (!mbar_wait(bar(L::FULL + slot), (u / NS) & 1, ab)) return false;
-                if (!mbar_wait(bar(L::S_FREE + sb), ((j >> 1) & 1) ^ 1, ab)) return false;
-                tc_fence_after();
-                const uint32_t ka = sbase + L::kOffRing + slot * kSlotBytes, qa = sbase + L::kOffQ;
+            // scores of a step with nt tiles whose operands start at ring position u0
+            auto issue_qk = [&](int ss_, int nt, int u0) -> bool {
+                const int set = ss_ & 1;
+                if (!mbar_wait(bar(L::S_FREE + set), ((ss_ >> 1) & 1) ^ 1, ab)) return false;
+                for (int i = 0; i < nt; ++i) {
+                    const int u = u0 + i, slot = u % NS;
+                    if (!mbar_wait(bar(L::FULL + slot), (u / NS) & 1, ab)) return false;
+                    tc_fence_after();
+                    const uint32_t ka = sbase + L::kOffRing + slot * kSlotBytes, qa = sbase + L::kOffQ;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    umma_bf16(tmem_s[sb], smem_desc(ka + (ks >> 2) * kHalfT + (ks & 3) * 32, 16, 1024),
-                              smem_desc(qa + (ks >> 2) * (NB * 128) + (ks & 3) * 32, 16, 1024), idesc_qk, ks > 0);
-                umma_commit(bar(L::EMPTY + slot));
-                umma_commit(bar(L::S_FULL + sb));
+                    for (int ks = 0; ks < 8; ++ks)
+                        umma_bf16(tmem + (uint32_t)((2 * set + i) * NB), smem_desc(ka + (ks >> 2) * 1024 + (ks & 3) * 32, 16, 2048),
+                                  smem_desc(qa + (ks >> 2) * (NB * 128) + (ks & 3) * 32, 16, 1024), idesc_qk, ks > 0);
+                    umma_commit(bar(L::EMPTY + slot));
+                }
+                umma_commit(bar(L::S_FULL + set));
                 return true;
             };
-            while (g < g_end && alive) {
-                const SegInfo seg = segment_of_tile(p, cum, g);
+            SegInfo seg = seg0;
+            for (int g = g_begin;;) {
                 const int t_first = g - seg.tile_begin, t_last = min(seg.n_tiles, g_end - seg.tile_begin);
-                const int n = t_last - t_first;
+                const int n_steps = ceil_div(t_last - t_first, 2);
                 alive = mbar_wait(bar(L::Q_FULL), piece & 1, ab);
                 if (!alive) break;
                 tc_fence_after();
-                alive = issue_qk(it);
-                for (int j = 0; j < n && alive; ++j) {
-                    if (j + 1 < n) { alive = issue_qk(it + j + 1); if (!alive) break; }
-                    const int cur = it + j, u = 2 * cur + 1, slot = u % NS, pb = cur & 1;
-                    alive = mbar_wait(bar(L::P_FULL + pb), (cur >> 1) & 1, ab) && mbar_wait(bar(L::FULL + slot), (u / NS) & 1, ab);
-                    if (!alive) break;
-                    tc_fence_after();
-                    const uint32_t va = sbase + L::kOffRing + slot * kSlotBytes, pa = sbase + L::kOffP + pb * L::kPBytes;
+                alive = issue_qk(ss, step_tiles(t_first, t_last, 0), u_qk);
+                if (alive && n_steps == 1) umma_commit(bar(L::Q_FREE));      // the piece's last read of Q is under way
+                for (int j = 0; j < n_steps && alive; ++j) {
+                    const int nt = step_tiles(t_first, t_last, j);
+                    const int u_v = u_qk + nt;                // this step's V tiles follow its K tiles
+                    u_qk += 2 * nt;
+                    if (j + 1 < n_steps) {
+                        alive = issue_qk(ss + j + 1, step_tiles(t_first, t_last, j + 1), u_qk);
+                        if (!alive) break;
+                        if (j + 2 == n_steps) umma_commit(bar(L::Q_FREE));
+                    }
+                    alive = mbar_wait(bar(L::P_FULL), (ss + j) & 1, ab);
+                    for (int i = 0; i < nt && alive; ++i) {
+                        const int u = u_v + i, slot = u % NS;
+                        alive = mbar_wait(bar(L::FULL + slot), (u / NS) & 1, ab);
+                        if (!alive) break;
+                        tc_fence_after();
+                        const uint32_t va = sbase + L::kOffRing + slot * kSlotBytes, pa = sbase + L::kOffP + i * L::kPBytes;
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)          // 16 tokens per step: V rows ks*16.., P^T 32-byte column step
-                        umma_bf16(tmem_o, smem_desc(va + ks * 2048, kHalfT, 1024),
-                                  smem_desc(pa + (ks >> 2) * (NB * 128) + (ks & 3) * 32, 16, 1024), idesc_pv,
-                                  (j > 0 || ks > 0) ? 1u : 0u);
-                    umma_commit(bar(L::EMPTY + slot));
-                    umma_commit(bar(L::P_FREE + pb));
+                        for (int ks = 0; ks < 8; ++ks)      // one page (16 tokens) per step; P^T 32-byte column step
+                            umma_bf16(tmem_o, smem_desc(va + ks * 4096, 1024, 2048),
+                                      smem_desc(pa + (ks >> 2) * (NB * 128) + (ks & 3) * 32, 16, 1024), idesc_pv,
+                                      (j > 0 || i > 0 || ks > 0) ? 1u : 0u);
+                        umma_commit(bar(L::EMPTY + slot));
+                    }
+                    if (alive) umma_commit(bar(L::P_FREE));
                 }
-                it += n; ++piece;
+                ss += n_steps; ++piece;
                 g = seg.tile_begin + t_last;
+                if (g >= g_end || !alive) break;
+                seg = next_segment(p, cum, seg);
             }
         }
     } else {
@@ -274,74 +325,99 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         // all softmax threads leave together.
         float* mref = reinterpret_cast<float*>(smem + L::kOffMref);
         float* red = reinterpret_cast<float*>(smem + L::kOffRed);
-        const unsigned long long* vis = reinterpret_cast<const unsigned long long*>(smem + L::kOffVis);
+        unsigned long long* vis = reinterpret_cast<unsigned long long*>(smem + L::kOffVis);
         const int quarter = warp & 3, cg = warp >> 2;       // TMEM lane quarter of this warp, column group
-        const int tok = quarter * 32 + lane;                 // this thread's token in the tile; its dim in O^T
+        const int tok = quarter * 32 + lane;                 // this thread's token in either tile; its dim in O^T
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         auto row_of = [&](int k) { return 4 * (cg + CG * k); };    // first row of this thread's k-th chunk
-        int it = 0;
+        int ss = 0, piece = 0, u0 = 0;                        // steps, pieces, operand tiles of this CTA so far
         bool ok = true;
-        SegInfo seg = segment_of_tile(p, cum, g_begin);
-        stage_q<NB, NT>(p, seg, smem, tid);
+        SegInfo seg = seg0;
+        QFetch<NB, NT> qf;
+        qf.load(p, seg, tid);
+        qf.store(smem + L::kOffQ, tid);
         fence_proxy_async();
-        mbar_arrive(bar(L::Q_FULL));
+        warp_arrive(bar(L::Q_FULL), lane);
 
         for (;;) {
             const int t_first = g_begin > seg.tile_begin ? g_begin - seg.tile_begin : 0;
             const int t_last = min(seg.n_tiles, g_end - seg.tile_begin);
+            const int n_steps = ceil_div(t_last - t_first, 2);
             const int Ltok = seg.n_tokens;
             const int tail0 = seg.kind == 1 ? Ltok - p.R : Ltok;     // first token that needs the row mask
             const int n_rows = seg.n_rows;                            // chunks starting at or past it are skipped
+            const int g_next = seg.tile_begin + t_last;
+            const bool have_next = g_next < g_end;
+            SegInfo next = seg;
+            if (have_next) {
+                next = next_segment(p, cum, seg);
+                qf.load(p, next, tid);                                // in flight while this piece is computed
+            }
             float l_part[NCK][4];
 #pragma unroll
             for (int k = 0; k < NCK; ++k)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) l_part[k][e] = 0.f;
             if (tid < NB) mref[tid] = -INFINITY;
-            bar_sync_softmax<NT>();
+            if (seg.kind == 1 && p.tree_parents != nullptr && tid < p.R) vis[tid] = row_visibility(p, seg.b, tid);
+            bar_sync_id<NT>(1);
 
-            for (int t = t_first; t < t_last; ++t, ++it) {
-                const int sb = it & 1, pb = it & 1;
-                const int tok0 = t * kTileT;
-                const bool need_mask = tok0 + kTileT > tail0;        // uniform: tile touches masked / missing tokens
-                ok = ok && mbar_wait(bar(L::S_FULL + sb), (it >> 1) & 1, ab);
-                float s[NCK][4];                                      // raw scores of this token
+            for (int j = 0; j < n_steps; ++j, ++ss) {
+                const int set = ss & 1;
+                const int t = t_first + 2 * j;
+                const int nt = min(2, t_last - t);                    // uniform: tiles of this step
+                const bool need_mask = (t + nt) * kTileT > tail0;    // uniform: the step touches masked / missing tokens
+                ok = ok && mbar_wait(bar(L::S_FULL + set), (ss >> 1) & 1, ab);
+                float s[2][NCK][4];                                   // raw scores of this thread's two tokens
 #pragma unroll
-                for (int k = 0; k < NCK; ++k)
+                for (int i = 0; i < 2; ++i)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) s[k][e] = 0.f;
+                    for (int k = 0; k < NCK; ++k)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) s[i][k][e] = 0.f;
                 if (ok) {
                     tc_fence_after();
 #pragma unroll
-                    for (int k = 0; k < NCK; ++k)
-                        if (row_of(k) < n_rows) tmem_ld4(tmem_s[sb] + lane_base + (uint32_t)row_of(k), s[k]);
+                    for (int i = 0; i < 2; ++i)
+                        if (i < nt) {
+#pragma unroll
+                            for (int k = 0; k < NCK; ++k)
+                                if (row_of(k) < n_rows) tmem_ld4(tmem + lane_base + (uint32_t)((2 * set + i) * NB + row_of(k)), s[i][k]);
+                        }
                     tmem_wait_ld();
                 }
                 tc_fence_before();
-                mbar_arrive(bar(L::S_FREE + sb));            // the scores are in registers: S^T may be overwritten
+                warp_arrive(bar(L::S_FREE + set), lane);     // the scores are in registers: S^T may be overwritten
 
-                unsigned long long rowmask = ~0ull;         // bit r: this thread's token is visible to row r
+                unsigned long long rowmask[2] = {~0ull, ~0ull};     // bit r: token i of this thread is visible to row r
+                if (nt < 2) rowmask[1] = 0ull;
                 if (need_mask) {
-                    const int j = tok0 + tok;
-                    if (j >= Ltok) rowmask = 0ull;
-                    else if (j >= tail0) {
-                        // token a of the last R: visible to query position i = (row0 + r) / G iff i >= a
-                        // (causal) or a is i or an ancestor of i (tree)
-                        const int a = j - tail0;
-                        if (p.tree_parents == nullptr) {
-                            const int sh = a * p.G - seg.row0;
-                            rowmask = sh <= 0 ? ~0ull : (sh >= 64 ? 0ull : ~0ull << sh);
-                        } else {
-                            rowmask = 0ull;
-                            for (int r = 0; r < NB; ++r) {
-                                const int i = (seg.row0 + r) / p.G;
-                                if (i < p.R && ((vis[i] >> a) & 1ull)) rowmask |= 1ull << r;
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        if (i >= nt) continue;
+                        const int jt = (t + i) * kTileT + tok;
+                        if (jt >= Ltok) rowmask[i] = 0ull;
+                        else if (jt >= tail0) {
+                            // token a of the last R: visible to query position i = (row0 + r) / G iff i >= a
+                            // (causal) or a is i or an ancestor of i (tree)
+                            const int a = jt - tail0;
+                            if (p.tree_parents == nullptr) {
+                                const int sh = a * p.G - seg.row0;
+                                rowmask[i] = sh <= 0 ? ~0ull : (sh >= 64 ? 0ull : ~0ull << sh);
+                            } else {
+                                unsigned long long m = 0ull;
+                                for (int r = 0; r < NB; ++r) {
+                                    const int qi = (seg.row0 + r) / p.G;
+                                    if (qi < p.R && ((vis[qi] >> a) & 1ull)) m |= 1ull << r;
+                                }
+                                rowmask[i] = m;
                             }
                         }
                     }
                 }
+                const bool masked = need_mask || nt < 2;             // uniform
                 // d = score * scale - reference (log2 units); masked entries are -inf
-                float d[NCK][4];
+                float d[2][NCK][4];
                 auto compute_d = [&]() -> float {
                     float mx = -INFINITY;
 #pragma unroll
@@ -350,33 +426,37 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                             const float4 m4 = *reinterpret_cast<const float4*>(mref + row_of(k));
                             const float mm[4] = {m4.x, m4.y, m4.z, m4.w};
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                float v = fmaf(s[k][e], p.scale_log2, -mm[e]);      // +inf while the reference is -inf
-                                if (need_mask && !((rowmask >> (row_of(k) + e)) & 1ull)) v = -INFINITY;
-                                d[k][e] = v;
-                                mx = fmaxf(mx, v);
-                            }
+                            for (int i = 0; i < 2; ++i)
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    float v = fmaf(s[i][k][e], p.scale_log2, -mm[e]);      // +inf while the reference is -inf
+                                    if (masked && !((rowmask[i] >> (row_of(k) + e)) & 1ull)) v = -INFINITY;
+                                    d[i][k][e] = v;
+                                    mx = fmaxf(mx, v);
+                                }
                         }
                     }
                     return mx;
                 };
                 const float dmax = compute_d();
-                if (bar_red_or<NT>(dmax > kLazy || !ok)) {
+                if (bar_red_or<NT>(1, dmax > kLazy || !ok)) {
                     // ---- rare: move the reference of every row to the running maximum ----
-                    if (bar_red_or<NT>(!ok)) goto done;
+                    if (bar_red_or<NT>(1, !ok)) goto done;
 #pragma unroll
                     for (int k = 0; k < NCK; ++k) {
                         if (row_of(k) < n_rows) {
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
-                                float v = s[k][e] * p.scale_log2;
-                                if (need_mask && !((rowmask >> (row_of(k) + e)) & 1ull)) v = -INFINITY;
+                                float v = -INFINITY;
+#pragma unroll
+                                for (int i = 0; i < 2; ++i)
+                                    if (!masked || ((rowmask[i] >> (row_of(k) + e)) & 1ull)) v = fmaxf(v, s[i][k][e] * p.scale_log2);
                                 const float wm = warp_max_f32(v);
                                 if (lane == 0) red[quarter * NB + row_of(k) + e] = wm;
                             }
                         }
                     }
-                    bar_sync_softmax<NT>();
+                    bar_sync_id<NT>(1);
                     float fac[NCK][4];
                     bool any_scale = false;
 #pragma unroll
@@ -396,9 +476,9 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                         }
                     }
                     // whether any row of any column group moved is a block-wide question
-                    if (t > t_first && bar_red_or<NT>(any_scale)) {
-                        ok = ok && mbar_wait(bar(L::P_FREE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, ab);   // P.V of the previous tile done
-                        if (bar_red_or<NT>(!ok)) goto done;
+                    if (j > 0 && bar_red_or<NT>(1, any_scale)) {
+                        ok = ok && mbar_wait(bar(L::P_FREE), (ss & 1) ^ 1, ab);      // P.V of the previous step done
+                        if (bar_red_or<NT>(1, !ok)) goto done;
                         tc_fence_after();
 #pragma unroll
                         for (int k = 0; k < NCK; ++k) {
@@ -414,36 +494,40 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                         tmem_wait_st();
                         tc_fence_before();
                     }
-                    bar_sync_softmax<NT>();                  // everyone has read the old references
+                    bar_sync_id<NT>(1);                       // everyone has read the old references
                     if (tid < NB && (tid & ~3) < n_rows)
                         mref[tid] = fmaxf(mref[tid], fmaxf(fmaxf(red[tid], red[NB + tid]), fmaxf(red[2 * NB + tid], red[3 * NB + tid])));
-                    bar_sync_softmax<NT>();
+                    bar_sync_id<NT>(1);
                     compute_d();
                 }
 
-                // ---- probabilities of this token for its rows -> P^T ----
-                ok = ok && mbar_wait(bar(L::P_FREE + pb), ((it >> 1) & 1) ^ 1, ab);      // P.V two tiles back done
+                // ---- probabilities of this thread's tokens for its rows -> P^T of either tile ----
+                ok = ok && mbar_wait(bar(L::P_FREE), (ss & 1) ^ 1, ab);      // P.V of the previous step done
                 {
-                    unsigned char* pbase = smem + L::kOffP + pb * L::kPBytes + (tok >> 6) * (NB * 128) + (tok & 7) * 2;
+                    unsigned char* pbase = smem + L::kOffP + (tok >> 6) * (NB * 128) + (tok & 7) * 2;
                     const int chunk = (tok & 63) >> 3;
 #pragma unroll
-                    for (int k = 0; k < NCK; ++k) {
-                        if (row_of(k) < n_rows) {
-                            float e4[4];
+                    for (int i = 0; i < 2; ++i) {
+                        if (i >= nt) continue;
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                e4[e] = ex2(d[k][e]);                 // masked entries: ex2(-inf) = 0
-                                l_part[k][e] += e4[e];
-                            }
-                            if (ok) {
-                                __nv_bfloat162 h0 = __floats2bfloat162_rn(e4[0], e4[1]), h1 = __floats2bfloat162_rn(e4[2], e4[3]);
-                                const uint32_t w0 = *reinterpret_cast<uint32_t*>(&h0), w1 = *reinterpret_cast<uint32_t*>(&h1);
-                                const int r = row_of(k);              // multiple of 4: r & 7 is 0 or 4
-                                unsigned char* q0 = pbase + r * 128;
-                                *reinterpret_cast<unsigned short*>(q0 + ((chunk ^ (r & 7)) << 4)) = (unsigned short)(w0 & 0xffffu);
-                                *reinterpret_cast<unsigned short*>(q0 + 128 + ((chunk ^ ((r + 1) & 7)) << 4)) = (unsigned short)(w0 >> 16);
-                                *reinterpret_cast<unsigned short*>(q0 + 256 + ((chunk ^ ((r + 2) & 7)) << 4)) = (unsigned short)(w1 & 0xffffu);
-                                *reinterpret_cast<unsigned short*>(q0 + 384 + ((chunk ^ ((r + 3) & 7)) << 4)) = (unsigned short)(w1 >> 16);
+                        for (int k = 0; k < NCK; ++k) {
+                            if (row_of(k) < n_rows) {
+                                float e4[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    e4[e] = ex2(d[i][k][e]);          // masked entries: ex2(-inf) = 0
+                                    l_part[k][e] += e4[e];
+                                }
+                                if (ok) {
+                                    __nv_bfloat162 h0 = __floats2bfloat162_rn(e4[0], e4[1]), h1 = __floats2bfloat162_rn(e4[2], e4[3]);
+                                    const uint32_t w0 = *reinterpret_cast<uint32_t*>(&h0), w1 = *reinterpret_cast<uint32_t*>(&h1);
+                                    const int r = row_of(k);          // multiple of 4: r & 7 is 0 or 4
+                                    unsigned char* q0 = pbase + i * L::kPBytes + r * 128;
+                                    *reinterpret_cast<unsigned short*>(q0 + ((chunk ^ (r & 7)) << 4)) = (unsigned short)(w0 & 0xffffu);
+                                    *reinterpret_cast<unsigned short*>(q0 + 128 + ((chunk ^ ((r + 1) & 7)) << 4)) = (unsigned short)(w0 >> 16);
+                                    *reinterpret_cast<unsigned short*>(q0 + 256 + ((chunk ^ ((r + 2) & 7)) << 4)) = (unsigned short)(w1 & 0xffffu);
+                                    *reinterpret_cast<unsigned short*>(q0 + 384 + ((chunk ^ ((r + 3) & 7)) << 4)) = (unsigned short)(w1 >> 16);
+                                }
                             }
                         }
                     }
@@ -451,36 +535,36 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 // last tile of a segment: V rows past the last valid token must be zero (they may hold
                 // anything, and 0 x NaN is NaN)
                 if (need_mask) {
-                    const int n_valid = min(kTileT, Ltok - tok0);
-                    if (n_valid < kTileT) {
-                        const int uv = 2 * it + 1, slot = uv % NS;
-                        ok = ok && mbar_wait(bar(L::FULL + slot), (uv / NS) & 1, ab);
-                        if (ok) {
-                            unsigned char* vb = smem + L::kOffRing + slot * kSlotBytes;
-                            for (int idx = tid; idx < (kTileT - n_valid) * 16; idx += NT) {
-                                const int row = n_valid + (idx >> 4), c = idx & 15;
-                                *reinterpret_cast<uint4*>(vb + (c >> 3) * kHalfT + row * 128 + ((c & 7) << 4)) = make_uint4(0, 0, 0, 0);
+                    for (int i = 0; i < nt; ++i) {
+                        const int n_valid = min(kTileT, Ltok - (t + i) * kTileT);
+                        if (n_valid < kTileT) {
+                            const int uv = u0 + nt + i, slot = uv % NS;
+                            ok = ok && mbar_wait(bar(L::FULL + slot), (uv / NS) & 1, ab);
+                            if (ok) {
+                                unsigned char* vb = smem + L::kOffRing + slot * kSlotBytes;
+                                for (int idx = tid; idx < (kTileT - n_valid) * 16; idx += NT) {
+                                    const int row = n_valid + (idx >> 4), c = idx & 15;
+                                    *reinterpret_cast<uint4*>(vb + tile_row_off(row) + (c >> 3) * 1024 + ((c & 7) << 4)) = make_uint4(0, 0, 0, 0);
+                                }
                             }
                         }
                     }
                 }
+                u0 += 2 * nt;
                 fence_proxy_async();
-                mbar_arrive(bar(L::P_FULL + pb));
+                warp_arrive(bar(L::P_FULL), lane);
             }
 
-            // ---- piece epilogue ----
-            const int g_next = seg.tile_begin + t_last;
-            const bool have_next = g_next < g_end;
-            SegInfo next = seg;
+            // ---- next piece's Q: its fetch is long done; store once this piece's last S^T is issued ----
             if (have_next) {
-                // all S^T of this piece have been seen, so its Q is no longer read: stage the next one now
-                next = segment_of_tile(p, cum, g_next);
-                stage_q<NB, NT>(p, next, smem, tid);
+                ok = ok && mbar_wait(bar(L::Q_FREE), piece & 1, ab);
+                if (ok) qf.store(smem + L::kOffQ, tid);
                 fence_proxy_async();
-                mbar_arrive(bar(L::Q_FULL));
+                warp_arrive(bar(L::Q_FULL), lane);
             }
-            ok = ok && mbar_wait(bar(L::P_FREE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, ab);      // last P.V done
-            if (bar_red_or<NT>(!ok)) goto done;
+            // ---- piece epilogue: partial (m, l, O) ----
+            ok = ok && mbar_wait(bar(L::P_FREE), (ss - 1) & 1, ab);          // last P.V done
+            if (bar_red_or<NT>(1, !ok)) goto done;
             tc_fence_after();
             {
                 float* po; float2* pml;
@@ -500,13 +584,14 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                         }
                     }
                 }
-                bar_sync_softmax<NT>();
+                bar_sync_id<NT>(1);
                 if (tid < n_rows)
                     pml[tid] = make_float2(mref[tid], (red[tid] + red[NB + tid]) + (red[2 * NB + tid] + red[3 * NB + tid]));
                 tc_fence_before();
-                bar_sync_softmax<NT>();
+                bar_sync_id<NT>(1);
             }
             if (!have_next) break;
+            ++piece;
             seg = next;
         }
     }
@@ -540,10 +625,10 @@ int umma_t_rows(int nr) { return nr <= 32 ? 32 : 64; }
 
 cudaError_t launch_attn_umma_t(Ctx* c, const AttnParams& p, cudaStream_t st) {
     cudaError_t err = cudaSuccess;
-    const CUtensorMap* mk = umma_pool_map(c, p.k_pages, &err);
+    const CUtensorMap* mk = umma_pool_map(c, p.k_pages, 1, &err);
     if (!mk) return err;
     const CUtensorMap mk_copy = *mk;                       // the cache may reallocate on the next insert
-    const CUtensorMap* mv = umma_pool_map(c, p.v_pages, &err);
+    const CUtensorMap* mv = umma_pool_map(c, p.v_pages, 1, &err);
     if (!mv) return err;
     if (p.rb_rows == 32) return launch_nb<32, 2>(c, p, mk_copy, *mv, st);
     if (p.rb_rows == 64) return launch_nb<64, 2>(c, p, mk_copy, *mv, st);

@@ -19,7 +19,7 @@ int cuda_fail(Ctx* c, cudaError_t e) {
 }
 
 // Row-block size and tile length the chosen kernel works with.
-struct Plan { int impl, rb_rows, tile_tokens, grid, copies; };
+struct Plan { int impl, rb_rows, tile_tokens, grid, copies, copies_pre; };
 
 Plan make_plan(const Ctx* c, int nr) {
     Plan pl;
@@ -29,13 +29,14 @@ Plan make_plan(const Ctx* c, int nr) {
     if (impl == TTS_ATTN_TCGEN05) impl = nr <= kUmmaTMaxRows ? TTS_ATTN_TCGEN05_TOKEN_MAJOR : TTS_ATTN_TCGEN05_ROW_MAJOR;
     pl.impl = impl;
     if (impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR) {
-        pl.rb_rows = umma_t_rows(nr); pl.tile_tokens = kUmmaTileTokens; pl.grid = c->n_sms; pl.copies = 1;
+        pl.rb_rows = umma_t_rows(nr); pl.tile_tokens = kUmmaTileTokens; pl.grid = c->n_sms;
+        pl.copies = pl.copies_pre = kUmmaTGroups;
     } else if (impl == TTS_ATTN_TCGEN05_ROW_MAJOR) {
         pl.rb_rows = kUmmaRows; pl.tile_tokens = kUmmaTileTokens; pl.grid = c->n_sms;
-        pl.copies = nr <= kUmmaRows ? umma_copies(nr) : 1;
+        pl.copies = nr <= kUmmaRows ? umma_copies(nr) : 1; pl.copies_pre = 1;
     } else {
         pl.rb_rows = simt_rb_rows(nr); pl.tile_tokens = kSimtTileTokens; pl.grid = c->n_sms * 3;
-        pl.copies = 1;
+        pl.copies = pl.copies_pre = 1;
     }
     return pl;
 }
@@ -47,10 +48,10 @@ void free_workspace(Ctx* c) {
 }
 
 // Partial-result rows one call needs: every piece reserves min(rb_rows, rows of its segment kind).
-void workspace_rows(int N, int Hkv, int nr, int rb_rows, int copies, int grid, size_t* pre, size_t* priv) {
+void workspace_rows(int N, int Hkv, int nr, int rb_rows, int copies, int copies_pre, int grid, size_t* pre, size_t* priv) {
     const long n_rb_pre = ((long)N * nr + rb_rows - 1) / rb_rows;
     const long n_rb_priv = (nr + rb_rows - 1) / rb_rows;
-    const long pre_stride = (long)N * nr < rb_rows ? (long)N * nr : rb_rows;
+    const long pre_stride = copies_pre * ((long)N * nr < rb_rows ? (long)N * nr : rb_rows);
     const long priv_stride = (long)copies * (nr < rb_rows ? nr : rb_rows);
     *pre = (size_t)(Hkv * n_rb_pre + grid) * pre_stride;
     *priv = (size_t)((long)N * Hkv * n_rb_priv + grid) * priv_stride;
@@ -62,15 +63,17 @@ cudaError_t alloc_workspace(Ctx* c) {
     const int G = f.n_q_heads / f.n_kv_heads;
     const int nr = f.max_rows_per_branch * G;
     size_t pre = 0, priv = 0;
-    const int cand_rb[5] = {8, 16, 32, 64, kUmmaRows};
-    for (int k = 0; k < 5; ++k) {
-        // a call may carry fewer rows than the maximum and then replicate them more often
-        for (int copies = 1; copies <= (k == 4 ? 4 : 1); copies *= 2) {
-            const int nr_c = copies == 1 ? nr : (nr < kUmmaRows / copies ? nr : kUmmaRows / copies);
-            size_t a, b;
-            workspace_rows(f.max_branches, f.n_kv_heads, nr_c, cand_rb[k], copies, c->n_sms * 3, &a, &b);
-            pre = a > pre ? a : pre; priv = b > priv ? b : priv;
-        }
+    // every (row block, copies of private pieces, copies of prefix pieces) a call may run with; a call
+    // may carry fewer rows than the maximum and the row-major kernel then replicates them more often
+    struct Cand { int rb, copies, copies_pre, nr_cap; };
+    const Cand cand[] = {{8, 1, 1, nr},  {16, 1, 1, nr}, {32, 1, 1, nr},                         // CUDA cores
+                         {32, kUmmaTGroups, kUmmaTGroups, nr}, {64, kUmmaTGroups, kUmmaTGroups, nr},   // token-major
+                         {kUmmaRows, 1, 1, nr}, {kUmmaRows, 2, 1, kUmmaRows / 2}, {kUmmaRows, 4, 1, kUmmaRows / 4}};
+    for (const Cand& k : cand) {
+        size_t a, b;
+        workspace_rows(f.max_branches, f.n_kv_heads, nr < k.nr_cap ? nr : k.nr_cap, k.rb, k.copies, k.copies_pre,
+                       c->n_sms * 3, &a, &b);
+        pre = a > pre ? a : pre; priv = b > priv ? b : priv;
     }
     cudaError_t e;
     if ((e = cudaMalloc(&c->part_o_pre, pre * kHeadDim * sizeof(float))) != cudaSuccess) return e;
@@ -102,7 +105,7 @@ int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
 
     {
         size_t need_pre, need_priv;
-        workspace_rows(n_branches, f.n_kv_heads, nr, pl.rb_rows, pl.copies, pl.grid, &need_pre, &need_priv);
+        workspace_rows(n_branches, f.n_kv_heads, nr, pl.rb_rows, pl.copies, pl.copies_pre, pl.grid, &need_pre, &need_priv);
         if (need_pre > c->pre_rows || need_priv > c->priv_rows) return TTS_ERR_INVALID;
     }
     cudaError_t e;
@@ -120,9 +123,9 @@ int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
     p.N = n_branches; p.R = rows; p.Hq = f.n_q_heads; p.Hkv = f.n_kv_heads; p.G = G; p.nr = nr;
     p.P = prefix_len; p.max_blocks = f.max_blocks_per_branch; p.num_pages = f.num_pages;
     p.rb_rows = pl.rb_rows;
-    p.pre_stride = n_branches * nr < pl.rb_rows ? n_branches * nr : pl.rb_rows;
+    p.pre_stride = pl.copies_pre * (n_branches * nr < pl.rb_rows ? n_branches * nr : pl.rb_rows);
     p.priv_stride = pl.copies * (nr < pl.rb_rows ? nr : pl.rb_rows);
-    p.copies = pl.copies;
+    p.copies = pl.copies; p.copies_pre = pl.copies_pre;
     p.n_rb_pre = ceil_div(n_branches * nr, pl.rb_rows);
     p.n_rb_priv = ceil_div(nr, pl.rb_rows);
     p.n_pre = prefix_len > 0 ? f.n_kv_heads * p.n_rb_pre : 0;

@@ -47,8 +47,9 @@ struct AttnParams {
     int P;                          // prefix tokens
     int max_blocks, num_pages;
     int rb_rows;                    // rows per row block
-    int pre_stride, priv_stride;    // rows reserved per piece: min(rb_rows, N*nr) / copies * min(rb_rows, nr)
-    int copies;                     // tcgen05 path: independent key-slice copies of a private piece's rows
+    int pre_stride, priv_stride;    // rows reserved per piece: copies_pre * min(rb_rows, N*nr) / copies * min(rb_rows, nr)
+    int copies;                     // tcgen05 paths: independent key-subset copies of a private piece's rows,
+    int copies_pre;                 //   and of a prefix piece's rows (each copy is a partial result of its own)
     int n_rb_pre, n_rb_priv;        // row blocks per prefix kv head / per (branch, kv head)
     int n_pre;                      // prefix segments (0 when P == 0)
     int tiles_pre;                  // tiles per prefix segment
@@ -60,6 +61,7 @@ struct AttnParams {
 
 struct SegInfo {
     int kind;        // 0 prefix, 1 private
+    int idx;         // group b*Hkv + kvh the segment belongs to (private) or follows (prefix)
     int kvh, rb, b;  // b = -1 for prefix
     int n_rows;      // valid rows in this row block
     int row0;        // first stacked row of the block (prefix: in [0, N*nr); private: in [0, nr))
@@ -114,9 +116,9 @@ __device__ inline int total_tiles(const AttnParams& p, const int* cum) {
     return group_tile_begin(p, cum, p.N * p.Hkv);
 }
 
-__device__ inline SegInfo prefix_segment(const AttnParams& p, int s, int tile_begin) {
+__device__ inline SegInfo prefix_segment(const AttnParams& p, int s, int tile_begin, int idx) {
     SegInfo g;
-    g.kind = 0; g.b = -1;
+    g.kind = 0; g.b = -1; g.idx = idx;
     g.kvh = s / p.n_rb_pre; g.rb = s % p.n_rb_pre;
     g.row0 = g.rb * p.rb_rows;
     g.n_rows = min(p.rb_rows, p.N * p.nr - g.row0);
@@ -139,16 +141,43 @@ __device__ inline SegInfo segment_of_tile(const AttnParams& p, const int* cum, i
     const int within = g - begin;
     if (within >= priv_tiles) {                 // one of the prefix segments that follow the group
         const int k = (within - priv_tiles) / p.tiles_pre;
-        return prefix_segment(p, pre_before(p, idx) + k, begin + priv_tiles + k * p.tiles_pre);
+        return prefix_segment(p, pre_before(p, idx) + k, begin + priv_tiles + k * p.tiles_pre, idx);
     }
     SegInfo s;
-    s.kind = 1; s.b = b; s.kvh = kvh;
+    s.kind = 1; s.b = b; s.kvh = kvh; s.idx = idx;
     s.rb = within / tb;
     s.row0 = s.rb * p.rb_rows;
     s.n_rows = min(p.rb_rows, p.nr - s.row0);
     s.tile_begin = begin + s.rb * tb; s.n_tiles = tb;
     s.tok_begin = p.P; s.n_tokens = p.branch_lens[b];
     return s;
+}
+
+// The segment after s in the tile list (the caller knows there is one): the next row block of the
+// same group, else the next prefix segment that follows the group, else the next non-empty group.
+__device__ inline SegInfo next_segment(const AttnParams& p, const int* cum, const SegInfo& s) {
+    const int end = s.tile_begin + s.n_tiles;
+    if (s.kind == 1 && s.rb + 1 < p.n_rb_priv) {
+        SegInfo n = s;
+        n.rb = s.rb + 1; n.row0 = n.rb * p.rb_rows; n.n_rows = min(p.rb_rows, p.nr - n.row0);
+        n.tile_begin = end;
+        return n;
+    }
+    int idx = s.idx;
+    const int k_next = s.kind == 1 ? pre_before(p, idx) : s.kvh * p.n_rb_pre + s.rb + 1;
+    if (k_next < pre_before(p, idx + 1)) return prefix_segment(p, k_next, end, idx);
+    for (++idx; idx < p.N * p.Hkv - 1; ++idx) {           // skip groups without tiles
+        const int b = idx / p.Hkv;
+        if (cum[b + 1] - cum[b] > 0 || pre_before(p, idx + 1) > pre_before(p, idx)) break;
+    }
+    const int b = idx / p.Hkv;
+    if (cum[b + 1] - cum[b] == 0) return prefix_segment(p, pre_before(p, idx), end, idx);
+    SegInfo n;
+    n.kind = 1; n.idx = idx; n.b = b; n.kvh = idx - b * p.Hkv; n.rb = 0;
+    n.row0 = 0; n.n_rows = min(p.rb_rows, p.nr);
+    n.tile_begin = end; n.n_tiles = cum[b + 1] - cum[b];
+    n.tok_begin = p.P; n.n_tokens = p.branch_lens[b];
+    return n;
 }
 
 // First tile of prefix segment s: it follows the first group idx with pre_before(idx + 1) > s.
@@ -232,6 +261,7 @@ int umma_copies(int nr);              // replication factor of a private piece's
 cudaError_t launch_attn_umma(Ctx* c, const AttnParams& p, cudaStream_t st);
 // token-major tcgen05 kernel (KV tokens on the MMA M dimension): row blocks of 32 or 64 stacked rows
 constexpr int kUmmaTMaxRows = 64;
+constexpr int kUmmaTGroups = 1;        // partial results a piece leaves per row
 int umma_t_rows(int nr);
 cudaError_t launch_attn_umma_t(Ctx* c, const AttnParams& p, cudaStream_t st);
 void umma_release(Ctx* c);

@@ -7,9 +7,9 @@
 
 namespace tts {
 
-// Tensor map (cached per context) over a K or V page pool, for 64-dim x 16-token boxes with
-// 128-byte swizzle.  Null on failure, with *err set.
-const CUtensorMap* umma_pool_map(Ctx* c, const void* pool, cudaError_t* err);
+// Tensor map (cached per context) over a K or V page pool, 128-byte swizzle: kind 0 for 64-dim x
+// 16-token boxes, kind 1 for whole page-head tiles.  Null on failure, with *err set.
+const CUtensorMap* umma_pool_map(Ctx* c, const void* pool, int kind, cudaError_t* err);
 
 namespace ptx {
 
@@ -71,6 +71,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+// one whole page-head tile through the 5-D view of the pool (see umma_pool_map, kind 1)
+__device__ __forceinline__ void tma_load_page(uint32_t dst, const CUtensorMap* map, int page_head, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %2, %2, %2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(0), "r"(page_head), "r"(bar) : "memory");
 }
 
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
