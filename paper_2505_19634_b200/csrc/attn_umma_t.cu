@@ -13,9 +13,11 @@
 // (256 tokens) per step: the latency chain of a step (MMA -> TMEM load -> consensus -> exp -> P^T
 // -> MMA) is paid once for both tiles, and every thread works on two independent tokens.
 //
-//   producer warp    per step arms the "full" barriers of the next ring slots with the byte counts and
-//                    issues the TMA copies of the K tiles, then of the V tiles: one 5-D box per page-head
-//                    tile (4 KiB), laid out so that the 8 pages of a tile form one MMA operand
+//   producer warps   one for K, one for V, each with its own ring of slots (K tiles are consumed as soon
+//                    as they land, V tiles wait for the softmax of their step, so one FIFO would block
+//                    behind its oldest V tile): per tile the warp arms the "full" barrier of the next slot
+//                    with the byte count and issues one 5-D TMA box per page-head tile (4 KiB), laid out
+//                    so that the 8 pages of a tile form one MMA operand
 //   MMA warp         one thread: S^T of the step's tiles into one of two pairs of TMEM buffers (the
 //                    next step's scores are computed while the softmax warps work on this one's),
 //                    O^T (+)= V^T P^T once P^T has been published; tcgen05.commit frees ring slots,
@@ -29,8 +31,9 @@
 //                    with warp redux + shared memory and O^T is rescaled in TMEM).  The result is
 //                    exact either way: l is accumulated against the same reference.  Row sums are kept
 //                    per thread and reduced once per piece.  The Q block of the next piece is
-//                    prefetched into registers and stored once the MMA issuer has signalled that the
-//                    current piece no longer reads Q.
+//                    prefetched into registers and stored during the last step of the current piece
+//                    (its scores being complete, Q is no longer read), so that the next piece's first
+//                    scores are computed while this piece finishes.
 //
 // Every wait is bounded.  A wait that runs out raises TTS_ERR_DEVICE_TIMEOUT; the softmax warps only
 // leave their loops on the result of a block-wide reduction, so no thread is left behind at a named
@@ -53,13 +56,14 @@ constexpr float kLazy = 8.f;                         // the reference moves when
 template <int NB>
 struct Lay {
     static constexpr int kSlots = NB == 32 ? 6 : 5;
+    static constexpr int kSlotsK = 2, kSlotsV = kSlots - kSlotsK;   // ring of K tiles, ring of V tiles
     static constexpr int kQBytes = NB * 256;         // two 64-dim K-blocks of NB rows x 128 B
     static constexpr int kPBytes = NB * 256;         // two 64-token K-blocks of NB rows x 128 B
     static constexpr int kOffQ = 0;
     static constexpr int kOffP = kQBytes;            // one buffer per tile of a step
     static constexpr int kOffRing = kOffP + 2 * kPBytes;
     static constexpr int kOffBar = kOffRing + kSlots * kSlotBytes;
-    static constexpr int kOffMisc = kOffBar + 24 * 8;            // 2 * kSlots + 8 barriers
+    static constexpr int kOffMisc = kOffBar + 24 * 8;            // 2 * kSlots + 7 barriers
     static constexpr int kOffMref = kOffMisc + 64;               // float[NB]
     static constexpr int kOffRed = kOffMref + NB * 4;            // float[4][NB]
     static constexpr int kOffVis = kOffRed + 4 * NB * 4;         // u64[64]
@@ -68,7 +72,7 @@ struct Lay {
     static constexpr uint32_t kTmemCols = NB == 32 ? 256 : 512;  // 2 pairs of S^T buffers + O^T, power of two
     // barrier indices
     static constexpr int FULL = 0, EMPTY = kSlots, S_FULL = 2 * kSlots, S_FREE = S_FULL + 2, P_FULL = S_FREE + 2,
-                         P_FREE = P_FULL + 1, Q_FULL = P_FREE + 1, Q_FREE = Q_FULL + 1;
+                         P_FREE = P_FULL + 1, Q_FULL = P_FREE + 1;
 };
 
 // reducing / plain named barrier `id` over NT threads
@@ -150,19 +154,38 @@ struct QFetch {
 // [token half][dim half][8 tokens][128 bytes].
 __device__ __forceinline__ int tile_row_off(int row) { return (row >> 4) * 4096 + ((row >> 3) & 1) * 2048 + (row & 7) * 128; }
 
-// Tiles of step `ss` of a piece whose tiles are [t_first, t_last): 1 or 2.
-__device__ __forceinline__ int step_tiles(int t_first, int t_last, int ss_local) {
-    return min(2, t_last - t_first - 2 * ss_local);
-}
+// Walks the steps (two tiles, one at the end of a piece with an odd count) of a CTA's run of the tile list.
+struct StepCursor {
+    SegInfo seg;
+    int t, t_last;      // first tile of the step and end of the piece, as tile indices inside the segment
+    int piece;          // pieces before this one
+    int g_end;
+    bool valid, first;  // first: first step of its piece
+    __device__ void init(const SegInfo& s0, int g_begin, int g_end_) {
+        seg = s0; g_end = g_end_; piece = 0; valid = true; first = true;
+        t = g_begin - s0.tile_begin; t_last = min(s0.n_tiles, g_end_ - s0.tile_begin);
+    }
+    __device__ int nt() const { return min(2, t_last - t); }
+    __device__ bool last() const { return t + 2 >= t_last; }        // last step of its piece
+    __device__ void advance(const AttnParams& p, const int* cum) {
+        t += 2; first = false;
+        if (t < t_last) return;
+        if (seg.tile_begin + t_last >= g_end) { valid = false; return; }
+        seg = next_segment(p, cum, seg);
+        t = 0; t_last = min(seg.n_tiles, g_end - seg.tile_begin);
+        ++piece; first = true;
+    }
+};
 
 template <int NB, int CG>
-__global__ void __launch_bounds__(128 * CG + 64, 1)
+__global__ void __launch_bounds__(128 * CG + 96, 1)
 attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v) {
     using L = Lay<NB>;
     constexpr int NS = L::kSlots;
     constexpr int NT = 128 * CG;                           // softmax threads
     constexpr int NCK = NB / 4 / CG;                       // 4-row chunks per thread
-    constexpr int kProducerWarp = 4 * CG, kMmaWarp = kProducerWarp + 1;
+    constexpr int NK = L::kSlotsK, NV = L::kSlotsV;
+    constexpr int kProducerWarp = 4 * CG, kMmaWarp = kProducerWarp + 2;   // producers: K, then V
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -185,7 +208,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         for (int i = 0; i < NS; ++i) { mbar_init(bar(L::FULL + i), 1); mbar_init(bar(L::EMPTY + i), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(bar(L::S_FULL + i), 1); mbar_init(bar(L::S_FREE + i), 4 * CG); }
         mbar_init(bar(L::P_FULL), 4 * CG); mbar_init(bar(L::P_FREE), 1);     // softmax warps arrive once per warp
-        mbar_init(bar(L::Q_FULL), 4 * CG); mbar_init(bar(L::Q_FREE), 1);
+        mbar_init(bar(L::Q_FULL), 4 * CG);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMmaWarp) {
@@ -201,56 +224,48 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     const uint32_t tmem_o = tmem + 4u * NB;
     const SegInfo seg0 = segment_of_tile(p, cum, g_begin);
 
-    if (warp == kProducerWarp) {
-        // =========================== producer ===========================
-        int u = 0;                                          // operand tiles issued by this CTA
+    if (warp == kProducerWarp || warp == kProducerWarp + 1) {
+        // =========================== producers ===========================
+        const int op = warp - kProducerWarp;                // 0: K tiles into slots [0, NK), 1: V tiles into [NK, NS)
+        const int ring0 = op == 0 ? 0 : NK, ring_n = op == 0 ? NK : NV;
+        const CUtensorMap* tm = op == 0 ? &tm_k : &tm_v;
+        int u = 0;                                          // tiles of this operand issued by this CTA
         bool alive = true;
-        SegInfo seg = seg0;
-        for (int g = g_begin;;) {
-            const int t_first = g - seg.tile_begin, t_last = min(seg.n_tiles, g_end - seg.tile_begin);
+        StepCursor cur;
+        for (cur.init(seg0, g_begin, g_end); cur.valid && alive; cur.advance(p, cum)) {
+            const SegInfo& seg = cur.seg;
             const int32_t* bt = p.block_table + (size_t)(seg.kind == 0 ? 0 : seg.b) * p.max_blocks;
-            for (int t = t_first; t < t_last && alive; t += 2) {
-                const int nt = min(2, t_last - t);
-                int n_pages[2] = {0, 0}, y[2] = {0, 0};
-                for (int i = 0; i < nt; ++i) {
-                    const int tok0 = (t + i) * kTileT;
-                    n_pages[i] = ceil_div(min(kTileT, seg.n_tokens - tok0), kPage);
-                    int page = 0;
-                    if (lane < n_pages[i]) {
-                        page = bt[(seg.tok_begin + tok0) / kPage + lane];
-                        if (p.debug && (page < 0 || page >= p.num_pages)) {
-                            atomicMin(p.status, (int)TTS_ERR_DEVICE_BOUNDS);
-                            page = 0;
-                        }
+            const int nt = cur.nt();
+            for (int i = 0; i < nt && alive; ++i, ++u) {
+                const int tok0 = (cur.t + i) * kTileT;
+                const int n_pages = ceil_div(min(kTileT, seg.n_tokens - tok0), kPage);
+                int page = 0;
+                if (lane < n_pages) {
+                    page = bt[(seg.tok_begin + tok0) / kPage + lane];
+                    if (p.debug && (page < 0 || page >= p.num_pages)) {
+                        atomicMin(p.status, (int)TTS_ERR_DEVICE_BOUNDS);
+                        page = 0;
                     }
-                    y[i] = page * p.Hkv + seg.kvh;             // page-head index
                 }
-                // ring order of a step: K tiles, then V tiles (the order the MMA issuer consumes them in)
-                for (int k = 0; k < 2 * nt && alive; ++k, ++u) {
-                    const int op = k / nt, i = k - op * nt;
-                    const int slot = u % NS;
-                    if (lane == 0) {
-                        alive = mbar_wait(bar(L::EMPTY + slot), ((u / NS) & 1) ^ 1, ab);
-                        if (alive) mbar_arrive_expect_tx(bar(L::FULL + slot), (uint32_t)n_pages[i] * 4096u);
-                    }
-                    alive = __shfl_sync(0xffffffffu, alive, 0);
-                    if (alive && lane < n_pages[i])
-                        tma_load_page(sbase + L::kOffRing + slot * kSlotBytes + lane * 4096, op == 0 ? &tm_k : &tm_v, y[i],
-                                      bar(L::FULL + slot));
+                const int slot = ring0 + u % ring_n;
+                if (lane == 0) {
+                    alive = mbar_wait(bar(L::EMPTY + slot), ((u / ring_n) & 1) ^ 1, ab);
+                    if (alive) mbar_arrive_expect_tx(bar(L::FULL + slot), (uint32_t)n_pages * 4096u);
                 }
+                alive = __shfl_sync(0xffffffffu, alive, 0);
+                if (alive && lane < n_pages)
+                    tma_load_page(sbase + L::kOffRing + slot * kSlotBytes + lane * 4096, tm, page * p.Hkv + seg.kvh,
+                                  bar(L::FULL + slot));
             }
-            g = seg.tile_begin + t_last;
-            if (g >= g_end || !alive) break;
-            seg = next_segment(p, cum, seg);
         }
         // Copies this warp started must have landed before the CTA may exit: the consumers wait on
         // the same phases in the normal case; after an abort wait for them here (bounded).
         if (*ab.flag && lane == 0) {
-            for (int back = 1; back <= NS && back <= u; ++back) {
+            for (int back = 1; back <= ring_n && back <= u; ++back) {
                 const int j = u - back;
-                const Abort quiet{misc + 2, p.status};       // do not re-raise; misc[2] is scratch
-                misc[2] = 0;
-                mbar_wait(bar(L::FULL + j % NS), (j / NS) & 1, quiet);
+                const Abort quiet{misc + 2 + op, p.status};  // do not re-raise; misc[2], misc[3] are scratch
+                misc[2 + op] = 0;
+                mbar_wait(bar(L::FULL + ring0 + j % ring_n), (j / ring_n) & 1, quiet);
             }
         }
     } else if (warp == kMmaWarp) {
@@ -258,16 +273,19 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         if (lane == 0) {
             constexpr uint32_t idesc_qk = instr_desc(kTileT, NB, false, false);
             constexpr uint32_t idesc_pv = instr_desc(kTileT, NB, true, false);
-            int ss = 0, piece = 0;                           // steps / pieces of this CTA so far
-            int u_qk = 0;                                    // ring position of the next step's first K tile
             bool alive = true;
-            // scores of a step with nt tiles whose operands start at ring position u0
-            auto issue_qk = [&](int ss_, int nt, int u0) -> bool {
-                const int set = ss_ & 1;
-                if (!mbar_wait(bar(L::S_FREE + set), ((ss_ >> 1) & 1) ^ 1, ab)) return false;
-                for (int i = 0; i < nt; ++i) {
-                    const int u = u0 + i, slot = u % NS;
-                    if (!mbar_wait(bar(L::FULL + slot), (u / NS) & 1, ab)) return false;
+            int n_q = 0, n_p = 0, u_k = 0, u_v = 0;           // steps scored / accumulated, K / V tiles consumed
+            // scores of the step under `c`
+            auto issue_qk = [&](const StepCursor& c) -> bool {
+                const int set = n_q & 1;
+                if (c.first) {                                // a new piece: its Q block must have been staged
+                    if (!mbar_wait(bar(L::Q_FULL), c.piece & 1, ab)) return false;
+                }
+                if (!mbar_wait(bar(L::S_FREE + set), ((n_q >> 1) & 1) ^ 1, ab)) return false;
+                const int nt = c.nt();
+                for (int i = 0; i < nt; ++i, ++u_k) {
+                    const int slot = u_k % NK;
+                    if (!mbar_wait(bar(L::FULL + slot), (u_k / NK) & 1, ab)) return false;
                     tc_fence_after();
                     const uint32_t ka = sbase + L::kOffRing + slot * kSlotBytes, qa = sbase + L::kOffQ;
 #pragma unroll
@@ -277,46 +295,41 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                     umma_commit(bar(L::EMPTY + slot));
                 }
                 umma_commit(bar(L::S_FULL + set));
+                ++n_q;
                 return true;
             };
-            SegInfo seg = seg0;
-            for (int g = g_begin;;) {
-                const int t_first = g - seg.tile_begin, t_last = min(seg.n_tiles, g_end - seg.tile_begin);
-                const int n_steps = ceil_div(t_last - t_first, 2);
-                alive = mbar_wait(bar(L::Q_FULL), piece & 1, ab);
-                if (!alive) break;
-                tc_fence_after();
-                alive = issue_qk(ss, step_tiles(t_first, t_last, 0), u_qk);
-                if (alive && n_steps == 1) umma_commit(bar(L::Q_FREE));      // the piece's last read of Q is under way
-                for (int j = 0; j < n_steps && alive; ++j) {
-                    const int nt = step_tiles(t_first, t_last, j);
-                    const int u_v = u_qk + nt;                // this step's V tiles follow its K tiles
-                    u_qk += 2 * nt;
-                    if (j + 1 < n_steps) {
-                        alive = issue_qk(ss + j + 1, step_tiles(t_first, t_last, j + 1), u_qk);
-                        if (!alive) break;
-                        if (j + 2 == n_steps) umma_commit(bar(L::Q_FREE));
-                    }
-                    alive = mbar_wait(bar(L::P_FULL), (ss + j) & 1, ab);
-                    for (int i = 0; i < nt && alive; ++i) {
-                        const int u = u_v + i, slot = u % NS;
-                        alive = mbar_wait(bar(L::FULL + slot), (u / NS) & 1, ab);
-                        if (!alive) break;
-                        tc_fence_after();
-                        const uint32_t va = sbase + L::kOffRing + slot * kSlotBytes, pa = sbase + L::kOffP + i * L::kPBytes;
+            auto issue_pv = [&](const StepCursor& c) -> bool {
+                if (!mbar_wait(bar(L::P_FULL), n_p & 1, ab)) return false;
+                const int nt = c.nt();
+                for (int i = 0; i < nt; ++i, ++u_v) {
+                    const int slot = NK + u_v % NV;
+                    if (!mbar_wait(bar(L::FULL + slot), (u_v / NV) & 1, ab)) return false;
+                    tc_fence_after();
+                    const uint32_t va = sbase + L::kOffRing + slot * kSlotBytes, pa = sbase + L::kOffP + i * L::kPBytes;
 #pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)      // one page (16 tokens) per step; P^T 32-byte column step
-                            umma_bf16(tmem_o, smem_desc(va + ks * 4096, 1024, 2048),
-                                      smem_desc(pa + (ks >> 2) * (NB * 128) + (ks & 3) * 32, 16, 1024), idesc_pv,
-                                      (j > 0 || i > 0 || ks > 0) ? 1u : 0u);
-                        umma_commit(bar(L::EMPTY + slot));
-                    }
-                    if (alive) umma_commit(bar(L::P_FREE));
+                    for (int ks = 0; ks < 8; ++ks)          // one page (16 tokens) per step; P^T 32-byte column step
+                        umma_bf16(tmem_o, smem_desc(va + ks * 4096, 1024, 2048),
+                                  smem_desc(pa + (ks >> 2) * (NB * 128) + (ks & 3) * 32, 16, 1024), idesc_pv,
+                                  (!c.first || i > 0 || ks > 0) ? 1u : 0u);
+                    umma_commit(bar(L::EMPTY + slot));
                 }
-                ss += n_steps; ++piece;
-                g = seg.tile_begin + t_last;
-                if (g >= g_end || !alive) break;
-                seg = next_segment(p, cum, seg);
+                umma_commit(bar(L::P_FREE));
+                ++n_p;
+                return true;
+            };
+            // the scores run one step ahead of the accumulation, across piece boundaries too
+            StepCursor cq, cp;
+            cq.init(seg0, g_begin, g_end); cp = cq;
+            alive = issue_qk(cq);
+            cq.advance(p, cum);
+            while (alive && cp.valid) {
+                if (cq.valid) {
+                    alive = issue_qk(cq);
+                    if (!alive) break;
+                    cq.advance(p, cum);
+                }
+                alive = issue_pv(cp);
+                cp.advance(p, cum);
             }
         }
     } else {
@@ -330,7 +343,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         const int tok = quarter * 32 + lane;                 // this thread's token in either tile; its dim in O^T
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         auto row_of = [&](int k) { return 4 * (cg + CG * k); };    // first row of this thread's k-th chunk
-        int ss = 0, piece = 0, u0 = 0;                        // steps, pieces, operand tiles of this CTA so far
+        int ss = 0, u_v = 0;                                  // steps and V tiles of this CTA so far
         bool ok = true;
         SegInfo seg = seg0;
         QFetch<NB, NT> qf;
@@ -388,6 +401,12 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 }
                 tc_fence_before();
                 warp_arrive(bar(L::S_FREE + set), lane);     // the scores are in registers: S^T may be overwritten
+                if (have_next && j == n_steps - 1) {
+                    // the piece's last scores are complete, so its Q is no longer read: stage the next piece's
+                    if (ok) qf.store(smem + L::kOffQ, tid);
+                    fence_proxy_async();
+                    warp_arrive(bar(L::Q_FULL), lane);
+                }
 
                 unsigned long long rowmask[2] = {~0ull, ~0ull};     // bit r: token i of this thread is visible to row r
                 if (nt < 2) rowmask[1] = 0ull;
@@ -538,8 +557,8 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                     for (int i = 0; i < nt; ++i) {
                         const int n_valid = min(kTileT, Ltok - (t + i) * kTileT);
                         if (n_valid < kTileT) {
-                            const int uv = u0 + nt + i, slot = uv % NS;
-                            ok = ok && mbar_wait(bar(L::FULL + slot), (uv / NS) & 1, ab);
+                            const int uv = u_v + i, slot = NK + uv % NV;
+                            ok = ok && mbar_wait(bar(L::FULL + slot), (uv / NV) & 1, ab);
                             if (ok) {
                                 unsigned char* vb = smem + L::kOffRing + slot * kSlotBytes;
                                 for (int idx = tid; idx < (kTileT - n_valid) * 16; idx += NT) {
@@ -550,18 +569,11 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                         }
                     }
                 }
-                u0 += 2 * nt;
+                u_v += nt;
                 fence_proxy_async();
                 warp_arrive(bar(L::P_FULL), lane);
             }
 
-            // ---- next piece's Q: its fetch is long done; store once this piece's last S^T is issued ----
-            if (have_next) {
-                ok = ok && mbar_wait(bar(L::Q_FREE), piece & 1, ab);
-                if (ok) qf.store(smem + L::kOffQ, tid);
-                fence_proxy_async();
-                warp_arrive(bar(L::Q_FULL), lane);
-            }
             // ---- piece epilogue: partial (m, l, O) ----
             ok = ok && mbar_wait(bar(L::P_FREE), (ss - 1) & 1, ab);          // last P.V done
             if (bar_red_or<NT>(1, !ok)) goto done;
@@ -591,7 +603,6 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 bar_sync_id<NT>(1);
             }
             if (!have_next) break;
-            ++piece;
             seg = next;
         }
     }
@@ -615,7 +626,7 @@ cudaError_t launch_nb(Ctx* c, const AttnParams& p, const CUtensorMap& mk, const 
         if (err != cudaSuccess) return err;
         if (c->device >= 0 && c->device < 64) attr_set[c->device] = true;
     }
-    attn_umma_t_kernel<NB, CG><<<p.grid, 128 * CG + 64, smem, st>>>(p, mk, mv);
+    attn_umma_t_kernel<NB, CG><<<p.grid, 128 * CG + 96, smem, st>>>(p, mk, mv);
     return cudaGetLastError();
 }
 
