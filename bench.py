@@ -283,7 +283,7 @@ def run_ours(args, shape):
         value = total_bytes / (ms * 1e-3) / 1e9
         layer_bytes = shape.unique_kv_bytes()
         roof = {"bound": "hbm", "achieved": None, "peak": peak, "unit": "GB/s", "frac": None, "traffic": None,
-                "peak_kind": f"of {peak_kind}", "kernel": "attention main kernel (one layer per launch)"}
+                "peak_kind": f"of {peak_kind}", "kernel": "attn_umma_t_kernel (token-major tcgen05 attention, one layer per launch)"}
         if main_us:
             roof["achieved"] = layer_bytes / (main_us * 1e-6) / 1e9
             roof["frac"] = roof["achieved"] / peak
@@ -321,8 +321,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="32b", choices=list(ti.CONFIGS))
+    ap.add_argument("--layers", type=int, default=0,
+                    help="run only this many layers of the config (small cases for profiler captures; "
+                         "the workload name says so)")
     args = ap.parse_args()
     shape = ti.CONFIGS[args.config]
+    if args.layers > 0:
+        shape = ti.with_branches(shape, n_layers=args.layers)
     if args.impl == "reference":
         run_reference(args, shape)
     else:
