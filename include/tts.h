@@ -43,7 +43,8 @@ typedef enum {
     TTS_ERR_UNSUPPORTED = -2,    /* head_dim != 128, page_size != 16, unknown mask_kind / option */
     TTS_ERR_CUDA = -3,           /* a CUDA call failed; tts_last_cuda_error() has the code */
     TTS_ERR_DEVICE_BOUNDS = -4,  /* (via tts_last_status) a kernel saw a page id / token out of range */
-    TTS_ERR_DEVICE_TIMEOUT = -5  /* (via tts_last_status) a bounded device-side wait ran out */
+    TTS_ERR_DEVICE_TIMEOUT = -5, /* (via tts_last_status) a bounded device-side wait ran out */
+    TTS_ERR_SCRATCH = -6         /* tts_verify_attn_noalloc: the problem needs more than the fixed scratch array */
 } tts_status;
 
 enum { TTS_MASK_CAUSAL = 0, TTS_MASK_TREE = 1 };
@@ -119,6 +120,36 @@ TTS_API int tts_verify_attn(tts_ctx* ctx, const void* q, const void* k_pages, co
 TTS_API int tts_verify_attn_tree(tts_ctx* ctx, const void* q, const void* k_pages, const void* v_pages,
                          const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
                          const int32_t* tree_parents, int n_branches, int n_nodes, void* out);
+
+/*
+ * Verify-step attention without any allocation (the paper has no counterpart: this entry point exists
+ * for the library's hosts, not for the method).  It is for callers that cannot obtain device memory
+ * when they call: a server that gave the whole GPU to its own pool allocator at start-up, a plugin
+ * inside a framework whose memory plan is frozen, code that must not trigger the implicit
+ * synchronisation of a driver allocation.  They cannot use tts_create (it calls cudaMalloc), so this
+ * function takes no context: shapes and the stream are arguments, and the split-KV partial results
+ * go to a fixed 8 MiB array inside the library image (each GPU that loads the library holds it
+ * until the process exits).  It computes exactly what tts_verify_attn computes with TTS_MASK_CAUSAL,
+ * bf16 output and scale 1/sqrt(128), on the CUDA-core kernel; it calls no cudaMalloc / cudaFree.
+ *   q, k_pages, v_pages, block_table, prefix_len, branch_lens, out: as for tts_verify_attn
+ *   max_blocks_per_branch: row stride of block_table; n_q_heads, n_kv_heads: as in tts_config
+ *   cuda_stream: cudaStream_t as void*, NULL = legacy default stream; the call is asynchronous on it
+ * Limits and caveats:
+ *   - a problem whose partial results exceed the array returns TTS_ERR_SCRATCH and launches nothing:
+ *     (Hkv * ceil(N*nr/rb) + 128) * min(N*nr, rb) + (N * Hkv * ceil(nr/rb) + 128) * min(nr, rb) rows of 520
+ *     bytes must fit 8 MiB, with nr = (gamma+1) * Hq/Hkv and rb = 8, 16 or 32 (the smallest >= nr, else 32);
+ *     the 32B-shaped layer (N 16, Hkv 8, nr 20) fits;
+ *   - the first call on a device looks up the array's address there (that device must be current);
+ *     make that first call before any stream capture;
+ *   - all calls share the one array, which keeps the previous call's contents (the status word in it
+ *     is cleared on the stream at every call; nothing else needs clearing); two calls whose kernels
+ *     may overlap on the GPU (different streams, no dependency) race on it - serialise them;
+ *   - device-side preconditions (page ids in range, branch_lens >= gamma+1) are not checked.
+ */
+TTS_API int tts_verify_attn_noalloc(const void* q, const void* k_pages, const void* v_pages,
+                            const int32_t* block_table, int max_blocks_per_branch, int prefix_len,
+                            const int32_t* branch_lens, int n_branches, int gamma, int n_q_heads,
+                            int n_kv_heads, void* out, void* cuda_stream);
 
 /*
  * Speculative-sampling accept / resample (the lossless verification rule of the works cited in

@@ -22,7 +22,7 @@ EXPORTED_SYMBOLS = (
     "tts_create", "tts_destroy", "tts_set_stream", "tts_verify_attn", "tts_verify_attn_tree",
     "tts_accept", "tts_majority_vote", "tts_confidence_max", "tts_greedy_search", "tts_last_status",
     "tts_last_cuda_error", "tts_launch_count", "tts_strerror", "tts_verify_step_host",
-    "tts_profile_enable", "tts_profile_read",
+    "tts_profile_enable", "tts_profile_read", "tts_verify_attn_noalloc",
 )
 
 
@@ -79,6 +79,7 @@ def load_library() -> ctypes.CDLL:
     lib.tts_strerror.restype = c_char_p
     lib.tts_verify_step_host.argtypes = [vp, c_int, vp, POINTER(c_void_p), POINTER(c_void_p), vp, c_int, vp,
                                          c_int, c_int, vp, vp, vp, vp, c_int, vp, vp, vp]
+    lib.tts_verify_attn_noalloc.argtypes = [vp, vp, vp, vp, c_int, c_int, vp, c_int, c_int, c_int, c_int, vp, vp]
     for name in EXPORTED_SYMBOLS:
         fn = getattr(lib, name)
         if name not in ("tts_launch_count", "tts_strerror"):
@@ -200,6 +201,22 @@ class TtsContext:
             _ptr(branch_lens_host), int(n_branches), int(gamma), _ptr(p_target_host), _ptr(q_draft_host),
             _ptr(draft_tokens_host), _ptr(uniforms_host), int(vocab), _ptr(out_host), _ptr(accepted_len_host),
             _ptr(next_token_host)), "tts_verify_step_host")
+
+
+def tts_verify_attn_noalloc(q, k_pages, v_pages, block_table, max_blocks_per_branch: int, prefix_len: int,
+                            branch_lens, n_branches: int, gamma: int, n_q_heads: int, n_kv_heads: int, out,
+                            stream=None):
+    """Causal verify attention for callers that may not allocate device memory (no context, no
+    cudaMalloc: the partial results live in a fixed array inside the library).  Raises TtsError with
+    status -6 when the problem does not fit that array."""
+    lib = load_library()
+    handle = stream if isinstance(stream, int) or stream is None else stream.cuda_stream
+    rc = lib.tts_verify_attn_noalloc(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(block_table),
+                                     int(max_blocks_per_branch), int(prefix_len), _ptr(branch_lens),
+                                     int(n_branches), int(gamma), int(n_q_heads), int(n_kv_heads), _ptr(out),
+                                     c_void_p(handle or 0))
+    if rc != 0:
+        raise TtsError(rc, "tts_verify_attn_noalloc")
 
 
 # -- host-only helpers (no context) -----------------------------------------------------------

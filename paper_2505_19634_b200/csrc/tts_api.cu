@@ -368,6 +368,7 @@ const char* tts_strerror(int status) {
         case TTS_ERR_CUDA: return "CUDA call failed";
         case TTS_ERR_DEVICE_BOUNDS: return "device-side bounds check failed";
         case TTS_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case TTS_ERR_SCRATCH: return "problem exceeds the fixed scratch array of the no-allocation entry point";
         default: return "unknown status";
     }
 }
