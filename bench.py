@@ -164,6 +164,21 @@ def workload_name(shape):
             f"gamma={shape.gamma}, page 16 (random permutation), vocab {shape.vocab}")
 
 
+def aggregate_over_ranks(ms: float, e2e_ms: float, launches: int, world: int, device):
+    """Replicas only: every rank runs the same step on its own data, so the job's time is the
+    slowest rank's (MAX) and its launch count the sum; the bytes are summed by the caller as
+    world x bytes of one replica.  Needs an initialised process group when world > 1."""
+    if world <= 1:
+        return ms, e2e_ms, launches
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms, e2e_ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    lt = torch.tensor([launches], device=device, dtype=torch.int64)
+    dist.all_reduce(lt)
+    return float(t[0]), float(t[1]), int(lt[0])
+
+
 def run_ours(args, shape):
     import torch
     import torch.distributed as dist
@@ -269,13 +284,7 @@ def run_ours(args, shape):
            h_t.numel() * 4 + h_u.numel() * 4)
     d2h = out_host.numel() * 2 + 8 * N
 
-    if world > 1:
-        t = torch.tensor([ms, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = float(t[0]), float(t[1])
-        lt = torch.tensor([launches], device=dev, dtype=torch.int64)
-        dist.all_reduce(lt)
-        launches = int(lt[0])
+    ms, e2e_ms, launches = aggregate_over_ranks(ms, e2e_ms, launches, world, dev)
 
     if rank == 0:
         peak, peak_kind = measured_peaks()
