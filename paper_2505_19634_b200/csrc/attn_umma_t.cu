@@ -34,6 +34,9 @@
 //                    prefetched into registers and stored during the last step of the current piece
 //                    (its scores being complete, Q is no longer read), so that the next piece's first
 //                    scores are computed while this piece finishes.
+//   epilogue warps   4 warps: thread = TMEM lane = head dim.  O^T is double-buffered by piece parity, so
+//                    the softmax warps go straight on to the next piece while these warps wait for the
+//                    piece's last accumulation, read O^T and write the piece's partial (m, l, O).
 //
 // Every wait is bounded.  A wait that runs out raises TTS_ERR_DEVICE_TIMEOUT; the softmax warps only
 // leave their loops on the result of a block-wide reduction, so no thread is left behind at a named
@@ -63,16 +66,19 @@ struct Lay {
     static constexpr int kOffP = kQBytes;            // one buffer per tile of a step
     static constexpr int kOffRing = kOffP + 2 * kPBytes;
     static constexpr int kOffBar = kOffRing + kSlots * kSlotBytes;
-    static constexpr int kOffMisc = kOffBar + 24 * 8;            // 2 * kSlots + 7 barriers
+    static constexpr int kOffMisc = kOffBar + 32 * 8;            // 2 * kSlots + 15 barriers
     static constexpr int kOffMref = kOffMisc + 64;               // float[NB]
     static constexpr int kOffRed = kOffMref + NB * 4;            // float[4][NB]
     static constexpr int kOffVis = kOffRed + 4 * NB * 4;         // u64[64]
-    static constexpr int kOffCum = kOffVis + 64 * 8;             // int[N + 1]
+    static constexpr int kOffLsum = kOffVis + 64 * 8;            // float[2][4][NB]: row sums of a finished piece
+    static constexpr int kOffMout = kOffLsum + 2 * 4 * NB * 4;   // float[2][NB]: its row references
+    static constexpr int kOffCum = kOffMout + 2 * NB * 4;        // int[N + 1]
     static constexpr int kFixedBytes = kOffCum + 1024;           // + slack for the manual 1024-B alignment
-    static constexpr uint32_t kTmemCols = NB == 32 ? 256 : 512;  // 2 pairs of S^T buffers + O^T, power of two
+    static constexpr uint32_t kTmemCols = NB == 32 ? 256 : 512;  // 2 pairs of S^T buffers + 2 O^T, power of two
     // barrier indices
     static constexpr int FULL = 0, EMPTY = kSlots, S_FULL = 2 * kSlots, S_FREE = S_FULL + 2, P_FULL = S_FREE + 2,
-                         P_FREE = P_FULL + 1, Q_FULL = P_FREE + 1;
+                         P_FREE = P_FULL + 1, Q_FULL = P_FREE + 1, O_FULL = Q_FULL + 1, O_FREE = O_FULL + 2,
+                         L_FULL = O_FREE + 2, L_FREE = L_FULL + 2;
 };
 
 // reducing / plain named barrier `id` over NT threads
@@ -178,14 +184,15 @@ struct StepCursor {
 };
 
 template <int NB, int CG>
-__global__ void __launch_bounds__(128 * CG + 96, 1)
+__global__ void __launch_bounds__(128 * CG + 224, 1)
 attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v) {
     using L = Lay<NB>;
     constexpr int NS = L::kSlots;
     constexpr int NT = 128 * CG;                           // softmax threads
     constexpr int NCK = NB / 4 / CG;                       // 4-row chunks per thread
     constexpr int NK = L::kSlotsK, NV = L::kSlotsV;
-    constexpr int kProducerWarp = 4 * CG, kMmaWarp = kProducerWarp + 2;   // producers: K, then V
+    constexpr int kEpilogueWarp = 4 * CG;                  // 4 warps, a multiple of 4 from the start: warp & 3 = TMEM quarter
+    constexpr int kProducerWarp = kEpilogueWarp + 4, kMmaWarp = kProducerWarp + 2;   // producers: K, then V
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -209,6 +216,10 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         for (int i = 0; i < 2; ++i) { mbar_init(bar(L::S_FULL + i), 1); mbar_init(bar(L::S_FREE + i), 4 * CG); }
         mbar_init(bar(L::P_FULL), 4 * CG); mbar_init(bar(L::P_FREE), 1);     // softmax warps arrive once per warp
         mbar_init(bar(L::Q_FULL), 4 * CG);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar(L::O_FULL + i), 1); mbar_init(bar(L::O_FREE + i), 4);
+            mbar_init(bar(L::L_FULL + i), 4 * CG); mbar_init(bar(L::L_FREE + i), 4);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMmaWarp) {
@@ -220,8 +231,8 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = (uint32_t)misc[1];
-    // S^T of tile i of step ss at columns [(2 (ss & 1) + i) NB, +NB); O^T at [4 NB, +NB)
-    const uint32_t tmem_o = tmem + 4u * NB;
+    // S^T of tile i of step ss at columns [(2 (ss & 1) + i) NB, +NB); O^T of piece pc at [(4 + (pc & 1)) NB, +NB)
+    const uint32_t tmem_o0 = tmem + 4u * NB;
     const SegInfo seg0 = segment_of_tile(p, cum, g_begin);
 
     if (warp == kProducerWarp || warp == kProducerWarp + 1) {
@@ -299,6 +310,10 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 return true;
             };
             auto issue_pv = [&](const StepCursor& c) -> bool {
+                const int ob = c.piece & 1;
+                if (c.first) {                                // the epilogue of two pieces ago has read this O^T buffer
+                    if (!mbar_wait(bar(L::O_FREE + ob), ((c.piece >> 1) & 1) ^ 1, ab)) return false;
+                }
                 if (!mbar_wait(bar(L::P_FULL), n_p & 1, ab)) return false;
                 const int nt = c.nt();
                 for (int i = 0; i < nt; ++i, ++u_v) {
@@ -308,12 +323,13 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                     const uint32_t va = sbase + L::kOffRing + slot * kSlotBytes, pa = sbase + L::kOffP + i * L::kPBytes;
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)          // one page (16 tokens) per step; P^T 32-byte column step
-                        umma_bf16(tmem_o, smem_desc(va + ks * 4096, 1024, 2048),
+                        umma_bf16(tmem_o0 + (uint32_t)(ob * NB), smem_desc(va + ks * 4096, 1024, 2048),
                                   smem_desc(pa + (ks >> 2) * (NB * 128) + (ks & 3) * 32, 16, 1024), idesc_pv,
                                   (!c.first || i > 0 || ks > 0) ? 1u : 0u);
                     umma_commit(bar(L::EMPTY + slot));
                 }
                 umma_commit(bar(L::P_FREE));
+                if (c.last()) umma_commit(bar(L::O_FULL + ob));   // the piece's O^T is complete
                 ++n_p;
                 return true;
             };
@@ -332,6 +348,43 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 cp.advance(p, cum);
             }
         }
+    } else if (warp >= kEpilogueWarp) {
+        // =========================== epilogue warps ===========================
+        const int et = tid - NT, quarter = warp & 3;
+        const int dim = quarter * 32 + lane;                 // this thread's TMEM lane = head dim
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        const float* lsum = reinterpret_cast<const float*>(smem + L::kOffLsum);
+        const float* mout = reinterpret_cast<const float*>(smem + L::kOffMout);
+        SegInfo seg = seg0;
+        bool alive = true;
+        for (int pc = 0, g = g_begin; alive; ++pc) {
+            const int t_last = min(seg.n_tiles, g_end - seg.tile_begin);
+            const int pb = pc & 1, n_rows = seg.n_rows;
+            float* po; float2* pml;
+            piece_slot(p, seg, blockIdx.x, po, pml);
+            alive = mbar_wait(bar(L::L_FULL + pb), (pc >> 1) & 1, ab) && mbar_wait(bar(L::O_FULL + pb), (pc >> 1) & 1, ab);
+            alive = __all_sync(0xffffffffu, alive);
+            if (!alive) break;
+            tc_fence_after();
+            for (int r0 = 0; r0 < n_rows; r0 += 4) {
+                float o[4];
+                tmem_ld4(tmem_o0 + (uint32_t)(pb * NB) + lane_base + (uint32_t)r0, o);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (r0 + e < n_rows) po[(size_t)(r0 + e) * kHeadDim + dim] = o[e];
+            }
+            if (et < n_rows) {
+                const float* ls = lsum + pb * 4 * NB + et;
+                pml[et] = make_float2(mout[pb * NB + et], (ls[0] + ls[NB]) + (ls[2 * NB] + ls[3 * NB]));
+            }
+            tc_fence_before();
+            warp_arrive(bar(L::O_FREE + pb), lane);
+            warp_arrive(bar(L::L_FREE + pb), lane);
+            g = seg.tile_begin + t_last;
+            if (g >= g_end) break;
+            seg = next_segment(p, cum, seg);
+        }
     } else {
         // =========================== softmax warps ===========================
         // A wait that fails only clears `ok`; loops are left on block-wide reductions of !ok so that
@@ -343,7 +396,9 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         const int tok = quarter * 32 + lane;                 // this thread's token in either tile; its dim in O^T
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         auto row_of = [&](int k) { return 4 * (cg + CG * k); };    // first row of this thread's k-th chunk
-        int ss = 0, u_v = 0;                                  // steps and V tiles of this CTA so far
+        float* lsum = reinterpret_cast<float*>(smem + L::kOffLsum);
+        float* mout = reinterpret_cast<float*>(smem + L::kOffMout);
+        int ss = 0, u_v = 0, pc = 0;                          // steps, V tiles and pieces of this CTA so far
         bool ok = true;
         SegInfo seg = seg0;
         QFetch<NB, NT> qf;
@@ -359,6 +414,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
             const int Ltok = seg.n_tokens;
             const int tail0 = seg.kind == 1 ? Ltok - p.R : Ltok;     // first token that needs the row mask
             const int n_rows = seg.n_rows;                            // chunks starting at or past it are skipped
+            const uint32_t tmem_o = tmem_o0 + (uint32_t)((pc & 1) * NB);
             const int g_next = seg.tile_begin + t_last;
             const bool have_next = g_next < g_end;
             SegInfo next = seg;
@@ -574,34 +630,25 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 warp_arrive(bar(L::P_FULL), lane);
             }
 
-            // ---- piece epilogue: partial (m, l, O) ----
-            ok = ok && mbar_wait(bar(L::P_FREE), (ss - 1) & 1, ab);          // last P.V done
-            if (bar_red_or<NT>(1, !ok)) goto done;
-            tc_fence_after();
+            // ---- end of the piece: hand its row sums and references to the epilogue warps ----
             {
-                float* po; float2* pml;
-                piece_slot(p, seg, blockIdx.x, po, pml);
+                const int pb = pc & 1;
+                ok = ok && mbar_wait(bar(L::L_FREE + pb), ((pc >> 1) & 1) ^ 1, ab);      // read by the epilogue two pieces ago
+                if (bar_red_or<NT>(1, !ok)) goto done;
 #pragma unroll
                 for (int k = 0; k < NCK; ++k) {
                     if (row_of(k) < n_rows) {
-                        float o[4];
-                        tmem_ld4(tmem_o + lane_base + (uint32_t)row_of(k), o);
-                        tmem_wait_ld();
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const int r = row_of(k) + e;
-                            if (r < n_rows) po[(size_t)r * kHeadDim + tok] = o[e];
                             const float ws = warp_sum_f32(l_part[k][e]);
-                            if (lane == 0) red[quarter * NB + r] = ws;
+                            if (lane == 0) lsum[(pb * 4 + quarter) * NB + row_of(k) + e] = ws;
                         }
                     }
                 }
-                bar_sync_id<NT>(1);
-                if (tid < n_rows)
-                    pml[tid] = make_float2(mref[tid], (red[tid] + red[NB + tid]) + (red[2 * NB + tid] + red[3 * NB + tid]));
-                tc_fence_before();
-                bar_sync_id<NT>(1);
+                if (tid < NB) mout[pb * NB + tid] = mref[tid];            // the same thread resets mref[tid] below
+                warp_arrive(bar(L::L_FULL + pb), lane);
             }
+            ++pc;
             if (!have_next) break;
             seg = next;
         }
@@ -626,7 +673,7 @@ cudaError_t launch_nb(Ctx* c, const AttnParams& p, const CUtensorMap& mk, const 
         if (err != cudaSuccess) return err;
         if (c->device >= 0 && c->device < 64) attr_set[c->device] = true;
     }
-    attn_umma_t_kernel<NB, CG><<<p.grid, 128 * CG + 96, smem, st>>>(p, mk, mv);
+    attn_umma_t_kernel<NB, CG><<<p.grid, 128 * CG + 224, smem, st>>>(p, mk, mv);
     return cudaGetLastError();
 }
 
