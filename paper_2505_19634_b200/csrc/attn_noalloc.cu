@@ -105,6 +105,7 @@ extern "C" int tts_verify_attn_noalloc(const void* q, const void* k_pages, const
     p.copies = 1; p.copies_pre = 1;
     p.n_rb_pre = (int)n_rb_pre; p.n_rb_priv = (int)n_rb_priv;
     p.n_pre = prefix_len > 0 ? n_kv_heads * p.n_rb_pre : 0;
+    if ((long long)n_branches * n_kv_heads * p.n_pre >= (1ll << 31)) return TTS_ERR_UNSUPPORTED;
     p.tile_tokens = kSimtTileTokens;
     p.tiles_pre = ceil_div(prefix_len, kSimtTileTokens);
     p.grid = kNoAllocGrid;

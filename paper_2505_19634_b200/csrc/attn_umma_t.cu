@@ -139,9 +139,9 @@ struct QFetch {
             const int idx = t + k * NT, r = idx >> 4, c = idx & 15;
             v[k] = make_uint4(0, 0, 0, 0);
             if (r < seg.n_rows) {
-                int row = seg.row0 + r, b = seg.b;
-                if (seg.kind == 0) { b = row / p.nr; row = row % p.nr; }
-                const int i = row / p.G, gq = row % p.G;
+                int row = seg.row0 + r, b = seg.b, i, gq;
+                if (seg.kind == 0) fast_divmod(row, p.nr, b, row);
+                fast_divmod(row, p.G, i, gq);
                 const __nv_bfloat16* src = p.q + (((size_t)b * p.R + i) * p.Hq + seg.kvh * p.G + gq) * kHeadDim;
                 v[k] = __ldg(reinterpret_cast<const uint4*>(src) + c);
             }
@@ -436,34 +436,6 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 const int t = t_first + 2 * j;
                 const int nt = min(2, t_last - t);                    // uniform: tiles of this step
                 const bool need_mask = (t + nt) * kTileT > tail0;    // uniform: the step touches masked / missing tokens
-                ok = ok && mbar_wait(bar(L::S_FULL + set), (ss >> 1) & 1, ab);
-                float s[2][NCK][4];                                   // raw scores of this thread's two tokens
-#pragma unroll
-                for (int i = 0; i < 2; ++i)
-#pragma unroll
-                    for (int k = 0; k < NCK; ++k)
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) s[i][k][e] = 0.f;
-                if (ok) {
-                    tc_fence_after();
-#pragma unroll
-                    for (int i = 0; i < 2; ++i)
-                        if (i < nt) {
-#pragma unroll
-                            for (int k = 0; k < NCK; ++k)
-                                if (row_of(k) < n_rows) tmem_ld4(tmem + lane_base + (uint32_t)((2 * set + i) * NB + row_of(k)), s[i][k]);
-                        }
-                    tmem_wait_ld();
-                }
-                tc_fence_before();
-                warp_arrive(bar(L::S_FREE + set), lane);     // the scores are in registers: S^T may be overwritten
-                if (have_next && j == n_steps - 1) {
-                    // the piece's last scores are complete, so its Q is no longer read: stage the next piece's
-                    if (ok) qf.store(smem + L::kOffQ, tid);
-                    fence_proxy_async();
-                    warp_arrive(bar(L::Q_FULL), lane);
-                }
-
                 unsigned long long rowmask[2] = {~0ull, ~0ull};     // bit r: token i of this thread is visible to row r
                 if (nt < 2) rowmask[1] = 0ull;
                 if (need_mask) {
@@ -491,20 +463,35 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                     }
                 }
                 const bool masked = need_mask || nt < 2;             // uniform
-                // d = score * scale - reference (log2 units); masked entries are -inf
+                ok = ok && mbar_wait(bar(L::S_FULL + set), (ss >> 1) & 1, ab);
+                if (ok) tc_fence_after();
+                // d = score * scale - reference (log2 units), or the scaled score itself (raw); masked entries
+                // are -inf.  The scores are read from TMEM each time (the rare second pass re-reads them), so
+                // they do not occupy registers beside d.
                 float d[2][NCK][4];
-                auto compute_d = [&]() -> float {
+                auto compute_d = [&](bool raw) -> float {
+                    if (ok) {
+#pragma unroll
+                        for (int i = 0; i < 2; ++i)
+                            if (i < nt) {
+#pragma unroll
+                                for (int k = 0; k < NCK; ++k)
+                                    if (row_of(k) < n_rows) tmem_ld4(tmem + lane_base + (uint32_t)((2 * set + i) * NB + row_of(k)), d[i][k]);
+                            }
+                        tmem_wait_ld();
+                    }
                     float mx = -INFINITY;
 #pragma unroll
                     for (int k = 0; k < NCK; ++k) {
                         if (row_of(k) < n_rows) {
-                            const float4 m4 = *reinterpret_cast<const float4*>(mref + row_of(k));
+                            float4 m4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (!raw) m4 = *reinterpret_cast<const float4*>(mref + row_of(k));
                             const float mm[4] = {m4.x, m4.y, m4.z, m4.w};
 #pragma unroll
                             for (int i = 0; i < 2; ++i)
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
-                                    float v = fmaf(s[i][k][e], p.scale_log2, -mm[e]);      // +inf while the reference is -inf
+                                    float v = fmaf(d[i][k][e], p.scale_log2, -mm[e]);      // +inf while the reference is -inf
                                     if (masked && !((rowmask[i] >> (row_of(k) + e)) & 1ull)) v = -INFINITY;
                                     d[i][k][e] = v;
                                     mx = fmaxf(mx, v);
@@ -513,20 +500,17 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                     }
                     return mx;
                 };
-                const float dmax = compute_d();
+                const float dmax = compute_d(false);
                 if (bar_red_or<NT>(1, dmax > kLazy || !ok)) {
                     // ---- rare: move the reference of every row to the running maximum ----
                     if (bar_red_or<NT>(1, !ok)) goto done;
+                    compute_d(true);
 #pragma unroll
                     for (int k = 0; k < NCK; ++k) {
                         if (row_of(k) < n_rows) {
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
-                                float v = -INFINITY;
-#pragma unroll
-                                for (int i = 0; i < 2; ++i)
-                                    if (!masked || ((rowmask[i] >> (row_of(k) + e)) & 1ull)) v = fmaxf(v, s[i][k][e] * p.scale_log2);
-                                const float wm = warp_max_f32(v);
+                                const float wm = warp_max_f32(fmaxf(d[0][k][e], d[1][k][e]));
                                 if (lane == 0) red[quarter * NB + row_of(k) + e] = wm;
                             }
                         }
@@ -573,7 +557,15 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                     if (tid < NB && (tid & ~3) < n_rows)
                         mref[tid] = fmaxf(mref[tid], fmaxf(fmaxf(red[tid], red[NB + tid]), fmaxf(red[2 * NB + tid], red[3 * NB + tid])));
                     bar_sync_id<NT>(1);
-                    compute_d();
+                    compute_d(false);
+                }
+                tc_fence_before();
+                warp_arrive(bar(L::S_FREE + set), lane);     // the scores have been consumed: S^T may be overwritten
+                if (have_next && j == n_steps - 1) {
+                    // the piece's last scores are complete, so its Q is no longer read: stage the next piece's
+                    if (ok) qf.store(smem + L::kOffQ, tid);
+                    fence_proxy_async();
+                    warp_arrive(bar(L::Q_FULL), lane);
                 }
 
                 // ---- probabilities of this thread's tokens for its rows -> P^T of either tile ----

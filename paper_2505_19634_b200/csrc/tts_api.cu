@@ -129,6 +129,7 @@ int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
     p.n_rb_pre = ceil_div(n_branches * nr, pl.rb_rows);
     p.n_rb_priv = ceil_div(nr, pl.rb_rows);
     p.n_pre = prefix_len > 0 ? f.n_kv_heads * p.n_rb_pre : 0;
+    if ((long long)n_branches * f.n_kv_heads * p.n_pre >= (1ll << 31)) return TTS_ERR_UNSUPPORTED;
     p.tile_tokens = pl.tile_tokens;
     p.tiles_pre = ceil_div(prefix_len, pl.tile_tokens);
     p.grid = pl.grid;

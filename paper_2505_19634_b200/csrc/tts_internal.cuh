@@ -101,8 +101,17 @@ __device__ inline void build_branch_tile_prefix(const AttnParams& p, int* cum) {
 }
 
 // prefix segments placed before group idx (idx in [0, N*Hkv])
+// (the host rejects calls whose N * Hkv * n_pre does not fit 31 bits)
 __device__ inline int pre_before(const AttnParams& p, int idx) {
-    return (int)((long long)idx * p.n_pre / (p.N * p.Hkv));
+    return (int)((unsigned)idx * (unsigned)p.n_pre / (unsigned)(p.N * p.Hkv));
+}
+
+// a / b and a % b for 0 <= a < 2^23, 0 < b: float estimate, corrected exactly (integer division by a
+// run-time divisor is an expensive instruction sequence)
+__device__ __forceinline__ void fast_divmod(int a, int b, int& q, int& r) {
+    q = __float2int_rz(__fdividef((float)a, (float)b));
+    r = a - q * b;
+    if (r < 0) { --q; r += b; } else if (r >= b) { ++q; r -= b; }
 }
 
 // global index of the first tile of group idx (idx == N*Hkv gives the total)
