@@ -203,13 +203,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Abort ab{misc, p.status};
 
-    build_branch_tile_prefix(p, cum);
-    const int total = total_tiles(p, cum);
-    const int tpc = ceil_div(total, p.grid);
-    const int g_begin = blockIdx.x * tpc;
-    const int g_end = min(total, g_begin + tpc);
-    if (g_begin >= g_end) return;                          // uniform: nothing to do for this CTA
-
+    // ---- set-up that needs no input first: barriers, TMEM, tensor-map prefetch; then the run of this CTA ----
     if (tid == 0) {
         misc[0] = 0;
         for (int i = 0; i < NS; ++i) { mbar_init(bar(L::FULL + i), 1); mbar_init(bar(L::EMPTY + i), 1); }
@@ -226,16 +220,26 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + L::kOffMisc + 4), "r"(L::kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    if (warp == kProducerWarp && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
+    if (warp == kProducerWarp + 1 && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
     fence_proxy_async();
     tc_fence_before();
-    __syncthreads();
+    build_branch_tile_prefix(p, cum);                      // synchronises the CTA
     tc_fence_after();
     const uint32_t tmem = (uint32_t)misc[1];
+    const int total = total_tiles(p, cum);
+    const int tpc = ceil_div(total, p.grid);
+    const int g_begin = blockIdx.x * tpc;
+    const int g_end = min(total, g_begin + tpc);
+    const bool has_work = g_begin < g_end;                 // uniform
     // S^T of tile i of step ss at columns [(2 (ss & 1) + i) NB, +NB); O^T of piece pc at [(4 + (pc & 1)) NB, +NB)
     const uint32_t tmem_o0 = tmem + 4u * NB;
-    const SegInfo seg0 = segment_of_tile(p, cum, g_begin);
+    SegInfo seg0;
+    if (has_work) seg0 = segment_of_tile(p, cum, g_begin);
 
-    if (warp == kProducerWarp || warp == kProducerWarp + 1) {
+    if (!has_work) {
+        // nothing to do for this CTA
+    } else if (warp == kProducerWarp || warp == kProducerWarp + 1) {
         // =========================== producers ===========================
         const int op = warp - kProducerWarp;                // 0: K tiles into slots [0, NK), 1: V tiles into [NK, NS)
         const int ring0 = op == 0 ? 0 : NK, ring_n = op == 0 ? NK : NV;
@@ -500,6 +504,25 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                     }
                     return mx;
                 };
+                if (j == 0) {
+                    // First step of a piece: take the maximum over the 64 tokens of the quarter-0 warps as the
+                    // reference of every row (any reference within the lazy margin of the true maximum is as
+                    // good), instead of going through the exact update below with nothing accumulated yet.
+                    compute_d(true);
+                    if (quarter == 0) {
+#pragma unroll
+                        for (int k = 0; k < NCK; ++k) {
+                            if (row_of(k) < n_rows) {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const float wm = warp_max_f32(fmaxf(d[0][k][e], d[1][k][e]));
+                                    if (lane == 0) mref[row_of(k) + e] = wm;
+                                }
+                            }
+                        }
+                    }
+                    bar_sync_id<NT>(1);
+                }
                 const float dmax = compute_d(false);
                 if (bar_red_or<NT>(1, dmax > kLazy || !ok)) {
                     // ---- rare: move the reference of every row to the running maximum ----
