@@ -21,45 +21,71 @@ __global__ void __launch_bounds__(kRowsPerBlock * 32) attn_combine_kernel(const 
     const int total = total_tiles(p, cum);
     const int tpc = ceil_div(total, p.grid);
 
-    float m_run = -INFINITY, l_run = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-
-    // rows of one piece: `n_copies` stacked blocks of `rows_in_block` rows; row r of every block
-    // belongs to this output row
-    auto merge = [&](const float* o_base, const float2* ml_base, int stride, int seg_local, int r0,
-                     int rows_in_block, int n_copies, int t_begin, int n_tiles) {
-        if (n_tiles <= 0) return;
-        const int c0 = t_begin / tpc, c1 = (t_begin + n_tiles - 1) / tpc;
-        for (int cc = c0 * n_copies; cc < (c1 + 1) * n_copies; ++cc) {
-            const int c = cc / n_copies, r = (cc % n_copies) * rows_in_block + r0;
-            const size_t id = (size_t)seg_local + c;
-            const float2 ml = ml_base[id * stride + r];
-            if (!(ml.y > 0.f)) continue;                  // piece saw no visible key for this row
-            const float4 o = *reinterpret_cast<const float4*>(
-                o_base + (id * stride + r) * kHeadDim + lane * 4);
-            const float m_new = fmaxf(m_run, ml.x);
-            const float a = (m_run == -INFINITY) ? 0.f : exp2f(m_run - m_new);
-            const float w = exp2f(ml.x - m_new);
-            acc.x = acc.x * a + o.x * w; acc.y = acc.y * a + o.y * w;
-            acc.z = acc.z * a + o.z * w; acc.w = acc.w * a + o.w * w;
-            l_run = l_run * a + ml.y * w;
-            m_run = m_new;
-        }
-    };
-
+    // The row's partial results: `n_copies` stacked blocks of `rows_in_block` rows per piece, row r of
+    // every block belongs to this output row; first the pieces of its prefix segment, then those of its
+    // private segment.  Lanes fetch the (m, l) of up to 32 partials at once; the O rows are then loaded
+    // back to back (their addresses do not depend on the weights).
+    struct Part { const float* o; const float2* ml; int stride, seg, r0, rows_in_block, n_copies, c0, n; };
+    Part part[2];
+    int n_kinds = 0;
     const int r_priv = i * p.G + gq;
     if (p.n_pre > 0) {
         const int pr = b * p.nr + r_priv;
         const int rb = pr / p.rb_rows, r = pr % p.rb_rows;
         const int seg = kvh * p.n_rb_pre + rb;
-        merge(p.part_o_pre, p.part_ml_pre, p.pre_stride, seg, r, min(p.rb_rows, p.N * p.nr - rb * p.rb_rows), p.copies_pre,
-              prefix_segment_tile_begin(p, cum, seg), p.tiles_pre);
+        const int t_begin = prefix_segment_tile_begin(p, cum, seg);
+        const int c0 = t_begin / tpc, c1 = (t_begin + p.tiles_pre - 1) / tpc;
+        part[n_kinds++] = Part{p.part_o_pre, p.part_ml_pre, p.pre_stride, seg, r, min(p.rb_rows, p.N * p.nr - rb * p.rb_rows),
+                               p.copies_pre, c0, (c1 - c0 + 1) * p.copies_pre};
     }
-    {
+    if (tiles_b > 0) {
         const int rb = r_priv / p.rb_rows, r = r_priv % p.rb_rows;
         const int seg = (b * p.Hkv + kvh) * p.n_rb_priv + rb;
-        merge(p.part_o_priv, p.part_ml_priv, p.priv_stride, seg, r, min(p.rb_rows, p.nr - rb * p.rb_rows), p.copies,
-              group_tile_begin(p, cum, b * p.Hkv + kvh) + rb * tiles_b, tiles_b);
+        const int t_begin = group_tile_begin(p, cum, b * p.Hkv + kvh) + rb * tiles_b;
+        const int c0 = t_begin / tpc, c1 = (t_begin + tiles_b - 1) / tpc;
+        part[n_kinds++] = Part{p.part_o_priv, p.part_ml_priv, p.priv_stride, seg, r, min(p.rb_rows, p.nr - rb * p.rb_rows),
+                               p.copies, c0, (c1 - c0 + 1) * p.copies};
+    }
+    const int np = (n_kinds > 0 ? part[0].n : 0) + (n_kinds > 1 ? part[1].n : 0);
+
+    float m_run = -INFINITY, l_run = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int base = 0; base < np; base += 32) {
+        int j = base + lane;
+        const float* o_row = p.part_o_priv;                  // any valid address for lanes without a partial
+        float2 ml = make_float2(-INFINITY, 0.f);
+        if (j < np) {
+            const Part& k = (n_kinds > 1 && j >= part[0].n) ? part[1] : part[0];
+            if (n_kinds > 1 && j >= part[0].n) j -= part[0].n;
+            const int c = k.c0 + j / k.n_copies, r = (j % k.n_copies) * k.rows_in_block + k.r0;
+            const size_t row = (size_t)(k.seg + c) * k.stride + r;
+            o_row = k.o + row * kHeadDim;
+            ml = k.ml[row];
+        }
+        const bool live = ml.y > 0.f;                       // else the piece saw no visible key for this row
+        float m_new = live ? ml.x : -INFINITY;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m_new = fmaxf(m_new, __shfl_xor_sync(0xffffffffu, m_new, o));
+        m_new = fmaxf(m_new, m_run);
+        const float a = (m_run == -INFINITY || m_new == -INFINITY) ? 0.f : exp2f(m_run - m_new);
+        const float w = live ? exp2f(ml.x - m_new) : 0.f;
+        float lw = ml.y * w;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) lw += __shfl_xor_sync(0xffffffffu, lw, o);
+        l_run = l_run * a + lw;
+        acc.x *= a; acc.y *= a; acc.z *= a; acc.w *= a;
+        m_run = m_new;
+        const int cnt = min(32, np - base);
+        const unsigned long long o_addr = reinterpret_cast<unsigned long long>(o_row);
+#pragma unroll 4
+        for (int jj = 0; jj < cnt; ++jj) {
+            const float wj = __shfl_sync(0xffffffffu, w, jj);
+            const float4 o = *(reinterpret_cast<const float4*>(__shfl_sync(0xffffffffu, o_addr, jj)) + lane);
+            if (wj > 0.f) {
+                acc.x = fmaf(o.x, wj, acc.x); acc.y = fmaf(o.y, wj, acc.y);
+                acc.z = fmaf(o.z, wj, acc.z); acc.w = fmaf(o.w, wj, acc.w);
+            }
+        }
     }
 
     const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
