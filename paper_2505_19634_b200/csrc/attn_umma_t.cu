@@ -26,7 +26,7 @@
 //                    rows are cut into chunks of 4; column group cg owns chunks cg, cg+CG, ... and a
 //                    thread holds the scores of its tokens for the rows of its chunks (chunks past the
 //                    piece's last row are skipped).  The running reference m of every row lives in
-//                    shared memory and only moves when some score exceeds it by more than 2^8
+//                    shared memory and only moves when some score exceeds it by more than 2^16
 //                    (consensus through a reducing named barrier; the exact row maximum is then found
 //                    with warp redux + shared memory and O^T is rescaled in TMEM).  The result is
 //                    exact either way: l is accumulated against the same reference.  Row sums are kept
@@ -54,7 +54,7 @@ using namespace ptx;
 
 constexpr int kTileT = kUmmaTileTokens;              // 128 tokens = MMA M
 constexpr int kSlotBytes = kTileT * kHeadDim * 2;    // one K or V tile: 32 KiB
-constexpr float kLazy = 8.f;                         // the reference moves when exceeded by 2^8
+constexpr float kLazy = 16.f;                        // the reference moves when exceeded by 2^16
 
 template <int NB>
 struct Lay {
@@ -504,26 +504,43 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                     }
                     return mx;
                 };
+                float dmax;
                 if (j == 0) {
-                    // First step of a piece: take the maximum over the 64 tokens of the quarter-0 warps as the
-                    // reference of every row (any reference within the lazy margin of the true maximum is as
-                    // good), instead of going through the exact update below with nothing accumulated yet.
+                    // First step of a piece: the reference of every row is simply the score of the step's
+                    // first token (of its two tiles); any reference within the lazy margin of the true
+                    // maximum is as good, and the exact update below catches the rest.
                     compute_d(true);
-                    if (quarter == 0) {
+                    if (quarter == 0 && lane == 0) {
 #pragma unroll
                         for (int k = 0; k < NCK; ++k) {
                             if (row_of(k) < n_rows) {
 #pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const float wm = warp_max_f32(fmaxf(d[0][k][e], d[1][k][e]));
-                                    if (lane == 0) mref[row_of(k) + e] = wm;
-                                }
+                                for (int e = 0; e < 4; ++e) mref[row_of(k) + e] = fmaxf(d[0][k][e], d[1][k][e]);
                             }
                         }
                     }
                     bar_sync_id<NT>(1);
+                    dmax = -INFINITY;
+#pragma unroll
+                    for (int k = 0; k < NCK; ++k) {
+                        if (row_of(k) < n_rows) {
+                            const float4 m4 = *reinterpret_cast<const float4*>(mref + row_of(k));
+                            const float mm[4] = {m4.x, m4.y, m4.z, m4.w};
+#pragma unroll
+                            for (int i = 0; i < 2; ++i)
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    // masked entries stay -inf; a row whose first token is masked has -inf as its
+                                    // reference: +inf here, resolved by the exact update
+                                    const float v = d[i][k][e] == -INFINITY ? -INFINITY : d[i][k][e] - mm[e];
+                                    d[i][k][e] = v;
+                                    dmax = fmaxf(dmax, v);
+                                }
+                        }
+                    }
+                } else {
+                    dmax = compute_d(false);
                 }
-                const float dmax = compute_d(false);
                 if (bar_red_or<NT>(1, dmax > kLazy || !ok)) {
                     // ---- rare: move the reference of every row to the running maximum ----
                     if (bar_red_or<NT>(1, !ok)) goto done;

@@ -101,22 +101,24 @@ __device__ inline void build_branch_tile_prefix(const AttnParams& p, int* cum) {
 }
 
 // prefix segments placed before group idx (idx in [0, N*Hkv])
-// (the host rejects calls whose N * Hkv * n_pre does not fit 31 bits)
-__device__ inline int pre_before(const AttnParams& p, int idx) {
-    return (int)((unsigned)idx * (unsigned)p.n_pre / (unsigned)(p.N * p.Hkv));
-}
-
-// a / b and a % b for 0 <= a < 2^23, 0 < b: float estimate, corrected exactly (integer division by a
-// run-time divisor is an expensive instruction sequence)
+// a / b and a % b for 0 <= a < 2^31 with a quotient below 2^22, 0 < b: float estimate, corrected
+// exactly (integer division by a run-time divisor is an expensive instruction sequence)
 __device__ __forceinline__ void fast_divmod(int a, int b, int& q, int& r) {
     q = __float2int_rz(__fdividef((float)a, (float)b));
     r = a - q * b;
-    if (r < 0) { --q; r += b; } else if (r >= b) { ++q; r -= b; }
+    while (r < 0) { --q; r += b; }
+    while (r >= b) { ++q; r -= b; }
 }
+__device__ __forceinline__ int fast_div(int a, int b) { int q, r; fast_divmod(a, b, q, r); return q; }
+
+// prefix segments placed before group idx (idx in [0, N*Hkv]); the host rejects calls whose
+// N * Hkv * n_pre does not fit 31 bits
+__device__ inline int pre_before(const AttnParams& p, int idx) { return fast_div(idx * p.n_pre, p.N * p.Hkv); }
 
 // global index of the first tile of group idx (idx == N*Hkv gives the total)
 __device__ inline int group_tile_begin(const AttnParams& p, const int* cum, int idx) {
-    const int b = idx / p.Hkv, kvh = idx - b * p.Hkv;
+    int b, kvh;
+    fast_divmod(idx, p.Hkv, b, kvh);
     const int tb = b < p.N ? cum[b + 1] - cum[b] : 0;
     return p.n_rb_priv * (p.Hkv * cum[b] + kvh * tb) + p.tiles_pre * pre_before(p, idx);
 }
@@ -143,18 +145,20 @@ __device__ inline SegInfo segment_of_tile(const AttnParams& p, const int* cum, i
         const int mid = (lo + hi + 1) >> 1;
         if (group_tile_begin(p, cum, mid) <= g) lo = mid; else hi = mid - 1;
     }
-    const int idx = lo, b = idx / p.Hkv, kvh = idx - b * p.Hkv;
+    const int idx = lo;
+    int b, kvh;
+    fast_divmod(idx, p.Hkv, b, kvh);
     const int begin = group_tile_begin(p, cum, idx);
     const int tb = cum[b + 1] - cum[b];
     const int priv_tiles = p.n_rb_priv * tb;
     const int within = g - begin;
     if (within >= priv_tiles) {                 // one of the prefix segments that follow the group
-        const int k = (within - priv_tiles) / p.tiles_pre;
+        const int k = fast_div(within - priv_tiles, p.tiles_pre);
         return prefix_segment(p, pre_before(p, idx) + k, begin + priv_tiles + k * p.tiles_pre, idx);
     }
     SegInfo s;
     s.kind = 1; s.b = b; s.kvh = kvh; s.idx = idx;
-    s.rb = within / tb;
+    s.rb = fast_div(within, tb);
     s.row0 = s.rb * p.rb_rows;
     s.n_rows = min(p.rb_rows, p.nr - s.row0);
     s.tile_begin = begin + s.rb * tb; s.n_tiles = tb;
