@@ -190,3 +190,38 @@ def test_debug_bounds_reports_bad_page_id_without_faulting():
     assert ctx.tts_last_status() == -4
     assert ctx.tts_last_status() == 0                     # reading clears it
     ctx.close()
+
+
+def _sampled_rows(case, n, seed):
+    s = case.shape
+    rng = np.random.default_rng(seed)
+    rows = np.stack([rng.integers(0, s.n_branches, n), rng.integers(0, s.rows_per_branch, n),
+                     rng.integers(0, s.n_q_heads, n)], axis=1).astype(np.int32)
+    # always include the first and last row of the first and last branch
+    rows[:4] = [[0, 0, 0], [0, s.gamma, s.n_q_heads - 1], [s.n_branches - 1, 0, 0],
+                [s.n_branches - 1, s.gamma, s.n_q_heads - 1]]
+    return rows
+
+
+def _check_sampled(case, impl, rows, what):
+    want = oracle_out(case, row_sel=rows)
+    got = run_attn(case, impl, debug=False)[rows[:, 0], rows[:, 1], rows[:, 2]]
+    assert_attn_close(got, want, what=what)
+
+
+def test_32b_layer_full_size_sampled_rows():
+    """One layer of the benchmark's workload at full size (16 x 4096 private + 512 prefix tokens, 258 MiB of
+    K/V), in the launch configuration bench.py times (automatic kernel choice, no debug checks), on 96
+    sampled output rows the oracle computes one by one."""
+    case = ti.make_attn_case(replace(ti.CONFIGS["32b"], n_layers=1), 0x5EED + 2)
+    _check_sampled(case, tts.ATTN_AUTO, _sampled_rows(case, 96, 1), "32b layer")
+
+
+@pytest.mark.parametrize("n,gamma", [(64, 1), (7, 5)])
+def test_sweep_points_full_lengths_sampled_rows(n, gamma):
+    """Points of the branch/length sweep at full lengths (ragged 1024..8192 private tokens, prefix
+    256..1024, random page permutation), sampled rows."""
+    shp = ti.sweep_shape(n, gamma, seed=100 + n)
+    case = ti.make_attn_case(shp, 100 + n)
+    ti.poison_unused_slots(case)
+    _check_sampled(case, tts.ATTN_AUTO, _sampled_rows(case, 64, 2), shp.name)
