@@ -291,7 +291,10 @@ def run_ours(args, shape):
         total_bytes = step_bytes * world
         value = total_bytes / (ms * 1e-3) / 1e9
         layer_bytes = shape.unique_kv_bytes()
-        roof = {"bound": "hbm", "achieved": None, "peak": peak, "unit": "GB/s", "frac": None, "traffic": None,
+        # DRAM read + write bytes of one launch of the dominant kernel, from the ncu capture summarised in
+        # profiles/attn_umma_t_kernel_32b_2layers.md (valid for the 32b workload and this kernel version only)
+        traffic = 279.3e6 if shape.name == "32b" else None
+        roof = {"bound": "hbm", "achieved": None, "peak": peak, "unit": "GB/s", "frac": None, "traffic": traffic,
                 "peak_kind": f"of {peak_kind}", "kernel": "attn_umma_t_kernel (token-major tcgen05 attention, one layer per launch)"}
         if main_us:
             roof["achieved"] = layer_bytes / (main_us * 1e-6) / 1e9
