@@ -309,8 +309,8 @@ def run_ours(args, shape):
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "us_per_layer": ms * 1e3 / L,
             "frac_of_hbm_peak": value / world / peak,
-            "config": {"workload": workload_name(shape), "l2": "inputs larger than L2: %.1f GiB of KV per step, one pool per layer"
-                       % (layer_bytes * L / 2**30), "bytes_per_step": step_bytes,
+            "config": {"workload": workload_name(shape), "l2": "inputs larger than L2: %.2f GiB of KV per step, one K/V pool per layer (for a one-layer "
+                             "config: that many independent copies of the layer)" % (layer_bytes * L / 2**30), "bytes_per_step": step_bytes,
                        "attn_impl": os.environ.get("TTS_BENCH_IMPL", "auto")},
             "clocks": clocks,
             "e2e": {"value": total_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
@@ -340,6 +340,10 @@ def main():
     shape = ti.CONFIGS[args.config]
     if args.layers > 0:
         shape = ti.with_branches(shape, n_layers=args.layers)
+    elif shape.n_layers == 1:
+        # a one-layer config fits L2 (126 MB): time a rotation over enough independent copies of the
+        # layer (own K/V/Q each) that the working set exceeds twice the L2
+        shape = ti.with_branches(shape, n_layers=-(-2 * 132_000_000 // shape.unique_kv_bytes()))
     if args.impl == "reference":
         run_reference(args, shape)
     else:

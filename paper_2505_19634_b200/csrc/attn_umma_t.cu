@@ -5,7 +5,7 @@
 // the KV tokens go on the MMA M dimension instead and both contractions are computed transposed:
 //     S^T[128 tokens x NB rows] = K[128 x 128] . Q^T        (A = K tile, B = Q block, both K-major)
 //     O^T[128 dims   x NB rows] = V^T[128 x 128] . P^T      (A = V tile as MN-major, B = P^T K-major)
-// NB is 32 or 64.  The operands K and V are the TMA-staged page tiles themselves; Q and P^T are
+// NB is 32 (the code is generic in it).  The operands K and V are the TMA-staged page tiles themselves; Q and P^T are
 // small (NB x 256 bytes), which leaves room for a ring of 5-6 operand tiles (32 KiB each) in shared
 // memory, the depth that hides HBM latency at 4 KiB page granularity.
 //
@@ -711,7 +711,10 @@ cudaError_t launch_nb(Ctx* c, const AttnParams& p, const CUtensorMap& mk, const 
 
 }  // namespace
 
-int umma_t_rows(int nr) { return nr <= 32 ? 32 : 64; }
+// Row blocks of 32 also when a branch carries up to 64 rows per KV head (two blocks, the second reading
+// the K/V tiles that the first left in L2): the 64-row instantiation holds twice the scores per thread
+// and spills at the 128 registers that 15 warps allow, which cost more than the second pass.
+int umma_t_rows(int nr) { (void)nr; return 32; }
 
 cudaError_t launch_attn_umma_t(Ctx* c, const AttnParams& p, cudaStream_t st) {
     cudaError_t err = cudaSuccess;
@@ -721,7 +724,6 @@ cudaError_t launch_attn_umma_t(Ctx* c, const AttnParams& p, cudaStream_t st) {
     const CUtensorMap* mv = umma_pool_map(c, p.v_pages, 1, &err);
     if (!mv) return err;
     if (p.rb_rows == 32) return launch_nb<32, 2>(c, p, mk_copy, *mv, st);
-    if (p.rb_rows == 64) return launch_nb<64, 2>(c, p, mk_copy, *mv, st);
     return cudaErrorInvalidValue;
 }
 
