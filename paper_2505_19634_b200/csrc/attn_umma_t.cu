@@ -246,6 +246,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         const CUtensorMap* tm = op == 0 ? &tm_k : &tm_v;
         int u = 0;                                          // tiles of this operand issued by this CTA
         bool alive = true;
+        const uint64_t stream_once = l2_policy_evict_first();
         StepCursor cur;
         for (cur.init(seg0, g_begin, g_end); cur.valid && alive; cur.advance(p, cum)) {
             const SegInfo& seg = cur.seg;
@@ -270,7 +271,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 alive = __shfl_sync(0xffffffffu, alive, 0);
                 if (alive && lane < n_pages)
                     tma_load_page(sbase + L::kOffRing + slot * kSlotBytes + lane * 4096, tm, page * p.Hkv + seg.kvh,
-                                  bar(L::FULL + slot));
+                                  bar(L::FULL + slot), stream_once);
             }
         }
         // Copies this warp started must have landed before the CTA may exit: the consumers wait on

@@ -73,11 +73,20 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 
+// L2 policy for data that is read once: such lines are the first to be evicted, so that a stream of
+// K/V pages larger than the L2 does not push out what every launch needs again (the kernels' own
+// instructions, page tables, queries, partial results).
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
 // one whole page-head tile through the 5-D view of the pool (see umma_pool_map, kind 1)
-__device__ __forceinline__ void tma_load_page(uint32_t dst, const CUtensorMap* map, int page_head, uint32_t bar) {
+__device__ __forceinline__ void tma_load_page(uint32_t dst, const CUtensorMap* map, int page_head, uint32_t bar, uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %2, %2, %2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(0), "r"(page_head), "r"(bar) : "memory");
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %2, %2, %2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(0), "r"(page_head), "r"(bar), "l"(policy) : "memory");
 }
 
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
