@@ -234,8 +234,9 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     const bool has_work = g_begin < g_end;                 // uniform
     // S^T of tile i of step ss at columns [(2 (ss & 1) + i) NB, +NB); O^T of piece pc at [(4 + (pc & 1)) NB, +NB)
     const uint32_t tmem_o0 = tmem + 4u * NB;
+    const int group0 = group_of_tile_block(p, cum, has_work ? g_begin : 0);         // synchronises the CTA
     SegInfo seg0;
-    if (has_work) seg0 = segment_of_tile(p, cum, g_begin);
+    if (has_work) seg0 = segment_in_group(p, cum, group0, g_begin);
 
     if (!has_work) {
         // nothing to do for this CTA

@@ -138,14 +138,9 @@ __device__ inline SegInfo prefix_segment(const AttnParams& p, int s, int tile_be
     return g;
 }
 
-// Segment that contains global tile g (0 <= g < total).
-__device__ inline SegInfo segment_of_tile(const AttnParams& p, const int* cum, int g) {
-    int lo = 0, hi = p.N * p.Hkv - 1;          // largest group whose first tile is <= g
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (group_tile_begin(p, cum, mid) <= g) lo = mid; else hi = mid - 1;
-    }
-    const int idx = lo;
+// Segment that contains global tile g (0 <= g < total), given the group idx it falls into (the
+// largest one whose first tile is <= g).
+__device__ inline SegInfo segment_in_group(const AttnParams& p, const int* cum, int idx, int g) {
     int b, kvh;
     fast_divmod(idx, p.Hkv, b, kvh);
     const int begin = group_tile_begin(p, cum, idx);
@@ -164,6 +159,33 @@ __device__ inline SegInfo segment_of_tile(const AttnParams& p, const int* cum, i
     s.tile_begin = begin + s.rb * tb; s.n_tiles = tb;
     s.tok_begin = p.P; s.n_tokens = p.branch_lens[b];
     return s;
+}
+
+// Segment that contains global tile g (0 <= g < total): binary search by one thread.
+__device__ inline SegInfo segment_of_tile(const AttnParams& p, const int* cum, int g) {
+    int lo = 0, hi = p.N * p.Hkv - 1;          // largest group whose first tile is <= g
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (group_tile_begin(p, cum, mid) <= g) lo = mid; else hi = mid - 1;
+    }
+    return segment_in_group(p, cum, lo, g);
+}
+
+// The search alone (the group of tile g) for a value of g that is uniform over the thread block,
+// called by all its threads: the candidates of a round are tested by one thread each, so the search
+// takes one round per factor of blockDim.x in the number of groups instead of one dependent step
+// per factor of two.
+__device__ inline int group_of_tile_block(const AttnParams& p, const int* cum, int g) {
+    int lo = 0, n = p.N * p.Hkv;               // the group is in [lo, lo + n); group lo begins at or before g
+    while (n > 1) {
+        const int stride = ceil_div(n, (int)blockDim.x);
+        const int idx = lo + (int)threadIdx.x * stride;
+        const int c = __syncthreads_count(idx < lo + n && group_tile_begin(p, cum, idx) <= g);   // >= 1: thread 0
+        const int end = lo + n;
+        lo += (c - 1) * stride;
+        n = min(stride, end - lo);
+    }
+    return lo;
 }
 
 // The segment after s in the tile list (the caller knows there is one): the next row block of the
