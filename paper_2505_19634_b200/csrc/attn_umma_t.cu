@@ -66,7 +66,7 @@ struct Lay {
     static constexpr int kOffP = kQBytes;            // one buffer per tile of a step
     static constexpr int kOffRing = kOffP + 2 * kPBytes;
     static constexpr int kOffBar = kOffRing + kSlots * kSlotBytes;
-    static constexpr int kOffMisc = kOffBar + 32 * 8;            // 2 * kSlots + 16 barriers
+    static constexpr int kOffMisc = kOffBar + 32 * 8;            // 2 * kSlots + 15 barriers
     static constexpr int kOffMref = kOffMisc + 64;               // float[NB]
     static constexpr int kOffRed = kOffMref + NB * 4;            // float[4][NB]
     static constexpr int kOffVis = kOffRed + 4 * NB * 4;         // u64[64]
@@ -78,7 +78,7 @@ struct Lay {
     // barrier indices
     static constexpr int FULL = 0, EMPTY = kSlots, S_FULL = 2 * kSlots, S_FREE = S_FULL + 2, P_FULL = S_FREE + 2,
                          P_FREE = P_FULL + 1, Q_FULL = P_FREE + 1, O_FULL = Q_FULL + 1, O_FREE = O_FULL + 2,
-                         L_FULL = O_FREE + 2, L_FREE = L_FULL + 2, Q_FREE = L_FREE + 2;
+                         L_FULL = O_FREE + 2, L_FREE = L_FULL + 2;
 };
 
 // reducing / plain named barrier `id` over NT threads
@@ -209,7 +209,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         for (int i = 0; i < NS; ++i) { mbar_init(bar(L::FULL + i), 1); mbar_init(bar(L::EMPTY + i), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(bar(L::S_FULL + i), 1); mbar_init(bar(L::S_FREE + i), 4 * CG); }
         mbar_init(bar(L::P_FULL), 4 * CG); mbar_init(bar(L::P_FREE), 1);     // softmax warps arrive once per warp
-        mbar_init(bar(L::Q_FULL), 4); mbar_init(bar(L::Q_FREE), 1);          // the epilogue warps stage Q
+        mbar_init(bar(L::Q_FULL), 4 * CG);
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(L::O_FULL + i), 1); mbar_init(bar(L::O_FREE + i), 4);
             mbar_init(bar(L::L_FULL + i), 4 * CG); mbar_init(bar(L::L_FREE + i), 4);
@@ -312,7 +312,6 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                     umma_commit(bar(L::EMPTY + slot));
                 }
                 umma_commit(bar(L::S_FULL + set));
-                if (c.last()) umma_commit(bar(L::Q_FREE));      // the piece's last scores: its Q block is no longer read
                 ++n_q;
                 return true;
             };
@@ -364,29 +363,11 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         const float* mout = reinterpret_cast<const float*>(smem + L::kOffMout);
         SegInfo seg = seg0;
         bool alive = true;
-        QFetch<NB, 128> qf;
-        qf.load(p, seg, et);
-        qf.store(smem + L::kOffQ, et);
-        fence_proxy_async();
-        warp_arrive(bar(L::Q_FULL), lane);
-        for (int pc = 0; alive; ++pc) {
+        for (int pc = 0, g = g_begin; alive; ++pc) {
             const int t_last = min(seg.n_tiles, g_end - seg.tile_begin);
             const int pb = pc & 1, n_rows = seg.n_rows;
             float* po; float2* pml;
             piece_slot(p, seg, blockIdx.x, po, pml);
-            // The Q block of the next piece: fetched now, stored as soon as this piece's last scores are
-            // complete, so that the next piece's first scores are computed while this piece finishes.
-            const bool have_next = seg.tile_begin + t_last < g_end;
-            SegInfo next = seg;
-            if (have_next) {
-                next = next_segment(p, cum, seg);
-                qf.load(p, next, et);
-                alive = __all_sync(0xffffffffu, mbar_wait(bar(L::Q_FREE), pc & 1, ab));
-                if (!alive) break;
-                qf.store(smem + L::kOffQ, et);
-                fence_proxy_async();
-                warp_arrive(bar(L::Q_FULL), lane);
-            }
             alive = mbar_wait(bar(L::L_FULL + pb), (pc >> 1) & 1, ab) && mbar_wait(bar(L::O_FULL + pb), (pc >> 1) & 1, ab);
             alive = __all_sync(0xffffffffu, alive);
             if (!alive) break;
@@ -406,8 +387,9 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
             tc_fence_before();
             warp_arrive(bar(L::O_FREE + pb), lane);
             warp_arrive(bar(L::L_FREE + pb), lane);
-            if (!have_next) break;
-            seg = next;
+            g = seg.tile_begin + t_last;
+            if (g >= g_end) break;
+            seg = next_segment(p, cum, seg);
         }
     } else {
         // =========================== softmax warps ===========================
@@ -425,6 +407,11 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         int ss = 0, u_v = 0, pc = 0;                          // steps, V tiles and pieces of this CTA so far
         bool ok = true;
         SegInfo seg = seg0;
+        QFetch<NB, NT> qf;
+        qf.load(p, seg, tid);
+        qf.store(smem + L::kOffQ, tid);
+        fence_proxy_async();
+        warp_arrive(bar(L::Q_FULL), lane);
 
         for (;;) {
             const int t_first = g_begin > seg.tile_begin ? g_begin - seg.tile_begin : 0;
@@ -434,7 +421,13 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
             const int tail0 = seg.kind == 1 ? Ltok - p.R : Ltok;     // first token that needs the row mask
             const int n_rows = seg.n_rows;                            // chunks starting at or past it are skipped
             const uint32_t tmem_o = tmem_o0 + (uint32_t)((pc & 1) * NB);
-            const bool have_next = seg.tile_begin + t_last < g_end;
+            const int g_next = seg.tile_begin + t_last;
+            const bool have_next = g_next < g_end;
+            SegInfo next = seg;
+            if (have_next) {
+                next = next_segment(p, cum, seg);
+                qf.load(p, next, tid);                                // in flight while this piece is computed
+            }
             float l_part[NCK][4];
 #pragma unroll
             for (int k = 0; k < NCK; ++k)
@@ -610,6 +603,12 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 }
                 tc_fence_before();
                 warp_arrive(bar(L::S_FREE + set), lane);     // the scores have been consumed: S^T may be overwritten
+                if (have_next && j == n_steps - 1) {
+                    // the piece's last scores are complete, so its Q is no longer read: stage the next piece's
+                    if (ok) qf.store(smem + L::kOffQ, tid);
+                    fence_proxy_async();
+                    warp_arrive(bar(L::Q_FULL), lane);
+                }
 
                 // ---- probabilities of this thread's tokens for its rows -> P^T of either tile ----
                 ok = ok && mbar_wait(bar(L::P_FREE), (ss & 1) ^ 1, ab);      // P.V of the previous step done
@@ -685,7 +684,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
             }
             ++pc;
             if (!have_next) break;
-            seg = next_segment(p, cum, seg);
+            seg = next;
         }
     }
 done:
