@@ -402,6 +402,19 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         const int tok = quarter * 32 + lane;                 // this thread's token in either tile; its dim in O^T
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         auto row_of = [&](int k) { return 4 * (cg + CG * k); };    // first row of this thread's k-th chunk
+        // Where this thread's probabilities go.  P^T of a tile is the K-major B operand: two 64-token
+        // blocks of NB rows x 128 bytes, 16-byte units XOR-swizzled with the row (r & 7).  The rows of
+        // chunk k are 4 (cg + CG k) + e, e < 4; with an even CG their r & 7 is 4 (cg & 1) + e whatever k
+        // is, so one address per e serves all chunks and both tiles with constant offsets.
+        static_assert(CG % 2 == 0, "P^T store addresses assume an even number of column groups");
+        uint32_t p_addr[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            p_addr[e] = sbase + L::kOffP + (tok >> 6) * (NB * 128) + (4 * cg + e) * 128 +
+                        (((((tok & 63) >> 3) ^ (4 * (cg & 1) + e))) << 4) + (tok & 7) * 2;
+        auto store_p = [&](int i, int k, int e, uint32_t half) {      // row 4 (cg + CG k) + e of tile i
+            asm volatile("st.shared.u16 [%0], %1;" ::"r"(p_addr[e] + (uint32_t)(i * L::kPBytes + k * (4 * CG * 128))), "h"((unsigned short)half) : "memory");
+        };
         float* lsum = reinterpret_cast<float*>(smem + L::kOffLsum);
         float* mout = reinterpret_cast<float*>(smem + L::kOffMout);
         int ss = 0, u_v = 0, pc = 0;                          // steps, V tiles and pieces of this CTA so far
@@ -613,8 +626,6 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 // ---- probabilities of this thread's tokens for its rows -> P^T of either tile ----
                 ok = ok && mbar_wait(bar(L::P_FREE), (ss & 1) ^ 1, ab);      // P.V of the previous step done
                 {
-                    unsigned char* pbase = smem + L::kOffP + (tok >> 6) * (NB * 128) + (tok & 7) * 2;
-                    const int chunk = (tok & 63) >> 3;
 #pragma unroll
                     for (int i = 0; i < 2; ++i) {
                         if (i >= nt) continue;
@@ -630,12 +641,8 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                                 if (ok) {
                                     __nv_bfloat162 h0 = __floats2bfloat162_rn(e4[0], e4[1]), h1 = __floats2bfloat162_rn(e4[2], e4[3]);
                                     const uint32_t w0 = *reinterpret_cast<uint32_t*>(&h0), w1 = *reinterpret_cast<uint32_t*>(&h1);
-                                    const int r = row_of(k);          // multiple of 4: r & 7 is 0 or 4
-                                    unsigned char* q0 = pbase + i * L::kPBytes + r * 128;
-                                    *reinterpret_cast<unsigned short*>(q0 + ((chunk ^ (r & 7)) << 4)) = (unsigned short)(w0 & 0xffffu);
-                                    *reinterpret_cast<unsigned short*>(q0 + 128 + ((chunk ^ ((r + 1) & 7)) << 4)) = (unsigned short)(w0 >> 16);
-                                    *reinterpret_cast<unsigned short*>(q0 + 256 + ((chunk ^ ((r + 2) & 7)) << 4)) = (unsigned short)(w1 & 0xffffu);
-                                    *reinterpret_cast<unsigned short*>(q0 + 384 + ((chunk ^ ((r + 3) & 7)) << 4)) = (unsigned short)(w1 >> 16);
+                                    store_p(i, k, 0, w0 & 0xffffu); store_p(i, k, 1, w0 >> 16);
+                                    store_p(i, k, 2, w1 & 0xffffu); store_p(i, k, 3, w1 >> 16);
                                 }
                             }
                         }
