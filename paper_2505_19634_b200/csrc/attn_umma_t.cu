@@ -43,6 +43,8 @@
 // barrier; in-flight copies are awaited (bounded) and TMEM is released before the CTA returns.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "tts_internal.cuh"
 #include "umma_ptx.cuh"
 
@@ -488,15 +490,15 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 // are -inf.  The scores are read from TMEM each time (the rare second pass re-reads them), so
                 // they do not occupy registers beside d.
                 float d[2][NCK][4];
-                auto compute_d = [&](bool raw) -> float {
+                // (with_mask: a step without masked tokens skips the tests; the columns of a missing second
+                // tile hold stale scores, which the mask turns into -inf)
+                auto compute_d = [&](bool raw, auto with_mask) -> float {
                     if (ok) {
 #pragma unroll
                         for (int i = 0; i < 2; ++i)
-                            if (i < nt) {
 #pragma unroll
-                                for (int k = 0; k < NCK; ++k)
-                                    if (row_of(k) < n_rows) tmem_ld4(tmem + lane_base + (uint32_t)((2 * set + i) * NB + row_of(k)), d[i][k]);
-                            }
+                            for (int k = 0; k < NCK; ++k)
+                                if (row_of(k) < n_rows) tmem_ld4(tmem + lane_base + (uint32_t)((2 * set + i) * NB + row_of(k)), d[i][k]);
                         tmem_wait_ld();
                     }
                     float mx = -INFINITY;
@@ -511,7 +513,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
                                     float v = fmaf(d[i][k][e], p.scale_log2, -mm[e]);      // +inf while the reference is -inf
-                                    if (masked && !((rowmask[i] >> (row_of(k) + e)) & 1ull)) v = -INFINITY;
+                                    if (decltype(with_mask)::value && !((rowmask[i] >> (row_of(k) + e)) & 1ull)) v = -INFINITY;
                                     d[i][k][e] = v;
                                     mx = fmaxf(mx, v);
                                 }
@@ -524,7 +526,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                     // First step of a piece: the reference of every row is simply the score of the step's
                     // first token (of its two tiles); any reference within the lazy margin of the true
                     // maximum is as good, and the exact update below catches the rest.
-                    compute_d(true);
+                    compute_d(true, std::true_type{});
                     if (quarter == 0 && lane == 0) {
 #pragma unroll
                         for (int k = 0; k < NCK; ++k) {
@@ -554,12 +556,12 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                         }
                     }
                 } else {
-                    dmax = compute_d(false);
+                    dmax = masked ? compute_d(false, std::true_type{}) : compute_d(false, std::false_type{});
                 }
                 if (bar_red_or<NT>(1, dmax > kLazy || !ok)) {
                     // ---- rare: move the reference of every row to the running maximum ----
                     if (bar_red_or<NT>(1, !ok)) goto done;
-                    compute_d(true);
+                    compute_d(true, std::true_type{});
 #pragma unroll
                     for (int k = 0; k < NCK; ++k) {
                         if (row_of(k) < n_rows) {
@@ -612,7 +614,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                     if (tid < NB && (tid & ~3) < n_rows)
                         mref[tid] = fmaxf(mref[tid], fmaxf(fmaxf(red[tid], red[NB + tid]), fmaxf(red[2 * NB + tid], red[3 * NB + tid])));
                     bar_sync_id<NT>(1);
-                    compute_d(false);
+                    compute_d(false, std::true_type{});
                 }
                 tc_fence_before();
                 warp_arrive(bar(L::S_FREE + set), lane);     // the scores have been consumed: S^T may be overwritten
@@ -627,8 +629,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 ok = ok && mbar_wait(bar(L::P_FREE), (ss & 1) ^ 1, ab);      // P.V of the previous step done
                 {
 #pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        if (i >= nt) continue;
+                    for (int i = 0; i < 2; ++i) {                  // a missing second tile gets zeros (nobody reads them)
 #pragma unroll
                         for (int k = 0; k < NCK; ++k) {
                             if (row_of(k) < n_rows) {
@@ -638,12 +639,10 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                                     e4[e] = ex2(d[i][k][e]);          // masked entries: ex2(-inf) = 0
                                     l_part[k][e] += e4[e];
                                 }
-                                if (ok) {
-                                    __nv_bfloat162 h0 = __floats2bfloat162_rn(e4[0], e4[1]), h1 = __floats2bfloat162_rn(e4[2], e4[3]);
-                                    const uint32_t w0 = *reinterpret_cast<uint32_t*>(&h0), w1 = *reinterpret_cast<uint32_t*>(&h1);
-                                    store_p(i, k, 0, w0 & 0xffffu); store_p(i, k, 1, w0 >> 16);
-                                    store_p(i, k, 2, w1 & 0xffffu); store_p(i, k, 3, w1 >> 16);
-                                }
+                                __nv_bfloat162 h0 = __floats2bfloat162_rn(e4[0], e4[1]), h1 = __floats2bfloat162_rn(e4[2], e4[3]);
+                                const uint32_t w0 = *reinterpret_cast<uint32_t*>(&h0), w1 = *reinterpret_cast<uint32_t*>(&h1);
+                                store_p(i, k, 0, w0 & 0xffffu); store_p(i, k, 1, w0 >> 16);
+                                store_p(i, k, 2, w1 & 0xffffu); store_p(i, k, 3, w1 >> 16);
                             }
                         }
                     }
