@@ -414,8 +414,8 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         for (int e = 0; e < 4; ++e)
             p_addr[e] = sbase + L::kOffP + (tok >> 6) * (NB * 128) + (4 * cg + e) * 128 +
                         (((((tok & 63) >> 3) ^ (4 * (cg & 1) + e))) << 4) + (tok & 7) * 2;
-        auto store_p = [&](int i, int k, int e, uint32_t half) {      // row 4 (cg + CG k) + e of tile i
-            asm volatile("st.shared.u16 [%0], %1;" ::"r"(p_addr[e] + (uint32_t)(i * L::kPBytes + k * (4 * CG * 128))), "h"((unsigned short)half) : "memory");
+        auto store_p = [&](int i, int k, int e, unsigned short v) {   // row 4 (cg + CG k) + e of tile i
+            asm volatile("st.shared.u16 [%0], %1;" ::"r"(p_addr[e] + (uint32_t)(i * L::kPBytes + k * (4 * CG * 128))), "h"(v) : "memory");
         };
         float* lsum = reinterpret_cast<float*>(smem + L::kOffLsum);
         float* mout = reinterpret_cast<float*>(smem + L::kOffMout);
@@ -639,10 +639,8 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                                     e4[e] = ex2(d[i][k][e]);          // masked entries: ex2(-inf) = 0
                                     l_part[k][e] += e4[e];
                                 }
-                                __nv_bfloat162 h0 = __floats2bfloat162_rn(e4[0], e4[1]), h1 = __floats2bfloat162_rn(e4[2], e4[3]);
-                                const uint32_t w0 = *reinterpret_cast<uint32_t*>(&h0), w1 = *reinterpret_cast<uint32_t*>(&h1);
-                                store_p(i, k, 0, w0 & 0xffffu); store_p(i, k, 1, w0 >> 16);
-                                store_p(i, k, 2, w1 & 0xffffu); store_p(i, k, 3, w1 >> 16);
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) store_p(i, k, e, __bfloat16_as_ushort(__float2bfloat16_rn(e4[e])));
                             }
                         }
                     }
