@@ -414,6 +414,8 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         for (int e = 0; e < 4; ++e)
             p_addr[e] = sbase + L::kOffP + (tok >> 6) * (NB * 128) + (4 * cg + e) * 128 +
                         (((((tok & 63) >> 3) ^ (4 * (cg & 1) + e))) << 4) + (tok & 7) * 2;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) asm volatile("" : "+r"(p_addr[e]));      // kept in registers, not recomputed at every store
         auto store_p = [&](int i, int k, int e, unsigned short v) {   // row 4 (cg + CG k) + e of tile i
             asm volatile("st.shared.u16 [%0], %1;" ::"r"(p_addr[e] + (uint32_t)(i * L::kPBytes + k * (4 * CG * 128))), "h"(v) : "memory");
         };
