@@ -103,7 +103,9 @@ __global__ void __launch_bounds__(kRowsPerBlock * 32) attn_combine_kernel(const 
 
 }  // namespace
 
-cudaError_t launch_attn_combine(const AttnParams& p, cudaStream_t st) {
+cudaError_t launch_attn_combine(const AttnParams& main_params, cudaStream_t st) {
+    AttnParams p = main_params;
+    p.lens_smem = 0;                     // this kernel's shared memory holds the tile prefix only (N + 1 ints)
     const int rows = p.N * p.R * p.Hq;
     attn_combine_kernel<<<ceil_div(rows, kRowsPerBlock), kRowsPerBlock * 32, (p.N + 1) * sizeof(int), st>>>(p);
     return cudaGetLastError();

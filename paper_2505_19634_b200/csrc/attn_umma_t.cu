@@ -74,7 +74,7 @@ struct Lay {
     static constexpr int kOffVis = kOffRed + 4 * NB * 4;         // u64[64]
     static constexpr int kOffLsum = kOffVis + 64 * 8;            // float[2][4][NB]: row sums of a finished piece
     static constexpr int kOffMout = kOffLsum + 2 * 4 * NB * 4;   // float[2][NB]: its row references
-    static constexpr int kOffCum = kOffMout + 2 * NB * 4;        // int[N + 1]
+    static constexpr int kOffCum = kOffMout + 2 * NB * 4;        // int[2 N + 1]: tile prefix, branch lengths
     static constexpr int kFixedBytes = kOffCum + 1024;           // + slack for the manual 1024-B alignment
     static constexpr uint32_t kTmemCols = NB == 32 ? 256 : 512;  // 2 pairs of S^T buffers + 2 O^T, power of two
     // barrier indices
@@ -248,6 +248,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         const int ring0 = op == 0 ? 0 : NK, ring_n = op == 0 ? NK : NV;
         const CUtensorMap* tm = op == 0 ? &tm_k : &tm_v;
         int u = 0;                                          // tiles of this operand issued by this CTA
+        int ring_pos = 0, ring_round = 0;                   // u % ring_n, (u / ring_n) & 1, kept without dividing
         bool alive = true;
         const uint64_t stream_once = l2_policy_evict_first();
         StepCursor cur;
@@ -266,15 +267,16 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                         page = 0;
                     }
                 }
-                const int slot = ring0 + u % ring_n;
+                const int slot = ring0 + ring_pos;
                 if (lane == 0) {
-                    alive = mbar_wait(bar(L::EMPTY + slot), ((u / ring_n) & 1) ^ 1, ab);
+                    alive = mbar_wait(bar(L::EMPTY + slot), ring_round ^ 1, ab);
                     if (alive) mbar_arrive_expect_tx(bar(L::FULL + slot), (uint32_t)n_pages * 4096u);
                 }
                 alive = __shfl_sync(0xffffffffu, alive, 0);
                 if (alive && lane < n_pages)
                     tma_load_page(sbase + L::kOffRing + slot * kSlotBytes + lane * 4096, tm, page * p.Hkv + seg.kvh,
                                   bar(L::FULL + slot), stream_once);
+                if (++ring_pos == ring_n) { ring_pos = 0; ring_round ^= 1; }
             }
         }
         // Copies this warp started must have landed before the CTA may exit: the consumers wait on
@@ -705,11 +707,11 @@ done:
 
 template <int NB, int CG>
 cudaError_t launch_nb(Ctx* c, const AttnParams& p, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t st) {
-    const int smem = Lay<NB>::kFixedBytes + (p.N + 1) * (int)sizeof(int);
+    const int smem = Lay<NB>::kFixedBytes + (2 * p.N + 1) * (int)sizeof(int);
     static bool attr_set[64] = {};                          // the attribute is per device
     if (c->device < 0 || c->device >= 64 || !attr_set[c->device]) {
         cudaError_t err = cudaFuncSetAttribute(attn_umma_t_kernel<NB, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               Lay<NB>::kFixedBytes + (kMaxBranches + 1) * (int)sizeof(int));
+                                               Lay<NB>::kFixedBytes + (2 * kUmmaTMaxBranches + 1) * (int)sizeof(int));
         if (err != cudaSuccess) return err;
         if (c->device >= 0 && c->device < 64) attr_set[c->device] = true;
     }

@@ -21,12 +21,13 @@ int cuda_fail(Ctx* c, cudaError_t e) {
 // Row-block size and tile length the chosen kernel works with.
 struct Plan { int impl, rb_rows, tile_tokens, grid, copies, copies_pre; };
 
-Plan make_plan(const Ctx* c, int nr) {
+Plan make_plan(const Ctx* c, int nr, int n_branches) {
     Plan pl;
     int impl = c->cfg.attn_impl;
     if (impl == TTS_ATTN_AUTO) impl = umma_available() && nr >= kUmmaMinRows ? TTS_ATTN_TCGEN05 : TTS_ATTN_SIMT;
     // few rows per KV head: KV tokens on the MMA M dimension; many (draft trees): query rows on M
-    if (impl == TTS_ATTN_TCGEN05) impl = nr <= kUmmaTMaxRows ? TTS_ATTN_TCGEN05_TOKEN_MAJOR : TTS_ATTN_TCGEN05_ROW_MAJOR;
+    if (impl == TTS_ATTN_TCGEN05)
+        impl = nr <= kUmmaTMaxRows && n_branches <= kUmmaTMaxBranches ? TTS_ATTN_TCGEN05_TOKEN_MAJOR : TTS_ATTN_TCGEN05_ROW_MAJOR;
     pl.impl = impl;
     if (impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR) {
         pl.rb_rows = umma_t_rows(nr); pl.tile_tokens = kUmmaTileTokens; pl.grid = c->n_sms;
@@ -101,7 +102,8 @@ int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
 
     const int G = f.n_q_heads / f.n_kv_heads;
     const int nr = rows * G;
-    const Plan pl = make_plan(c, nr);
+    const Plan pl = make_plan(c, nr, n_branches);
+    if (pl.impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR && n_branches > kUmmaTMaxBranches) return TTS_ERR_UNSUPPORTED;   // only when asked for by name
 
     {
         size_t need_pre, need_priv;
@@ -133,6 +135,7 @@ int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
     p.tile_tokens = pl.tile_tokens;
     p.tiles_pre = ceil_div(prefix_len, pl.tile_tokens);
     p.grid = pl.grid;
+    p.lens_smem = pl.impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR ? 1 : 0;
     p.out_dtype = f.out_dtype; p.debug = f.debug_bounds;
     const float scale = f.softmax_scale > 0.f ? f.softmax_scale : 1.0f / sqrtf((float)f.head_dim);
     p.scale_log2 = scale * 1.4426950408889634f;

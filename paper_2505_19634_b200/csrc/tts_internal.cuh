@@ -56,6 +56,7 @@ struct AttnParams {
     int tile_tokens;
     int grid;                       // CTAs of the main kernel
     int out_dtype, debug;
+    int lens_smem;                  // the kernel keeps the branch lengths behind cum[] in shared memory (2N + 1 ints)
     float scale_log2;               // softmax scale * log2(e)
 };
 
@@ -74,10 +75,12 @@ struct SegInfo {
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 // cum[b] = tiles of branches < b (per private segment of that branch), cum[N] = sum.
-// Must be called by all threads of the block; cum lives in shared memory (N+1 ints).
+// Must be called by all threads of the block; cum lives in shared memory (N+1 ints, followed by
+// the N branch lengths themselves when p.lens_smem is set: the schedule then needs no global load).
 __device__ inline void build_branch_tile_prefix(const AttnParams& p, int* cum) {
     for (int b = threadIdx.x; b < p.N; b += blockDim.x) {
         int L = p.branch_lens[b];
+        if (p.lens_smem) cum[p.N + 1 + b] = L;
         L = L < 0 ? 0 : L;
         cum[b + 1] = ceil_div(L, p.tile_tokens);
     }
@@ -100,7 +103,10 @@ __device__ inline void build_branch_tile_prefix(const AttnParams& p, int* cum) {
     __syncthreads();
 }
 
-// prefix segments placed before group idx (idx in [0, N*Hkv])
+__device__ __forceinline__ int branch_len(const AttnParams& p, const int* cum, int b) {
+    return p.lens_smem ? cum[p.N + 1 + b] : p.branch_lens[b];
+}
+
 // a / b and a % b for 0 <= a < 2^31 with a quotient below 2^22, 0 < b: float estimate, corrected
 // exactly (integer division by a run-time divisor is an expensive instruction sequence)
 __device__ __forceinline__ void fast_divmod(int a, int b, int& q, int& r) {
@@ -157,7 +163,7 @@ __device__ inline SegInfo segment_in_group(const AttnParams& p, const int* cum, 
     s.row0 = s.rb * p.rb_rows;
     s.n_rows = min(p.rb_rows, p.nr - s.row0);
     s.tile_begin = begin + s.rb * tb; s.n_tiles = tb;
-    s.tok_begin = p.P; s.n_tokens = p.branch_lens[b];
+    s.tok_begin = p.P; s.n_tokens = branch_len(p, cum, b);
     return s;
 }
 
@@ -211,7 +217,7 @@ __device__ inline SegInfo next_segment(const AttnParams& p, const int* cum, cons
     n.kind = 1; n.idx = idx; n.b = b; n.kvh = idx - b * p.Hkv; n.rb = 0;
     n.row0 = 0; n.n_rows = min(p.rb_rows, p.nr);
     n.tile_begin = end; n.n_tiles = cum[b + 1] - cum[b];
-    n.tok_begin = p.P; n.n_tokens = p.branch_lens[b];
+    n.tok_begin = p.P; n.n_tokens = branch_len(p, cum, b);
     return n;
 }
 
@@ -296,6 +302,7 @@ int umma_copies(int nr);              // replication factor of a private piece's
 cudaError_t launch_attn_umma(Ctx* c, const AttnParams& p, cudaStream_t st);
 // token-major tcgen05 kernel (KV tokens on the MMA M dimension): row blocks of 32 or 64 stacked rows
 constexpr int kUmmaTMaxRows = 64;
+constexpr int kUmmaTMaxBranches = 896;   // its shared memory holds 2N + 1 schedule words beside the operand ring
 constexpr int kUmmaTGroups = 1;        // partial results a piece leaves per row
 int umma_t_rows(int nr);
 cudaError_t launch_attn_umma_t(Ctx* c, const AttnParams& p, cudaStream_t st);
