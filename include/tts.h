@@ -53,7 +53,8 @@ enum { TTS_OUT_BF16 = 0, TTS_OUT_FP32 = 1 };
  * stacked query rows per KV head make it worthwhile and CUDA cores otherwise.  TCGEN05 picks
  * between the two tensor-core kernels: TOKEN_MAJOR (KV tokens on the MMA M dimension, for at most
  * 64 rows per branch and KV head: chains of gamma+1 positions) and ROW_MAJOR (query rows on M, for
- * draft trees with many nodes).  The last two force one of them. */
+ * draft trees with many nodes).  The last two force one of them; TOKEN_MAJOR takes at most 896
+ * branches per call (TTS_ERR_UNSUPPORTED beyond; AUTO and TCGEN05 then use ROW_MAJOR). */
 enum { TTS_ATTN_AUTO = 0, TTS_ATTN_SIMT = 1, TTS_ATTN_TCGEN05 = 2, TTS_ATTN_TCGEN05_TOKEN_MAJOR = 3,
        TTS_ATTN_TCGEN05_ROW_MAJOR = 4 };
 

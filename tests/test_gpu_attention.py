@@ -71,6 +71,20 @@ def test_edge_shapes(impl, name):
     assert_attn_close(run_attn(case, impl), oracle_out(case), what=name)
 
 
+def test_more_branches_than_the_token_major_kernel_takes():
+    """Above 896 branches the token-major kernel's shared memory cannot hold the schedule: AUTO and
+    TCGEN05 go to the row-major kernel, asking for TOKEN_MAJOR by name is refused."""
+    n = 900
+    shp = replace(SMALL, n_branches=n, gamma=2, prefix_len=16, branch_lens=tuple(3 + (7 * i) % 23 for i in range(n)))
+    case = ti.make_attn_case(shp, 11)
+    want = oracle_out(case)
+    for impl in (tts.ATTN_AUTO, tts.ATTN_TCGEN05):
+        assert_attn_close(run_attn(case, impl), want, what=f"900 branches impl {impl}")
+    with pytest.raises(tts.TtsError) as e:
+        run_attn(case, tts.ATTN_TCGEN05_TOKEN_MAJOR)
+    assert e.value.status == -2                        # TTS_ERR_UNSUPPORTED
+
+
 @impl_param
 def test_sentinel_in_masked_positions(impl):
     """Enormous K/V in every position a row must not see: one leaked key changes out by O(1)."""
