@@ -1,6 +1,7 @@
 // Merge of the split-KV partial results: for every output row, the log-sum-exp combination of
 // the pieces of its prefix segment and of its private segment, normalisation and the cast to
 // the output type.  One warp per output row, four head dims per lane.
+#include "attn_merge.cuh"
 #include "tts_internal.cuh"
 
 namespace tts {
@@ -101,11 +102,31 @@ __global__ void __launch_bounds__(kRowsPerBlock * 32) attn_combine_kernel(const 
     }
 }
 
+// The same merge for the common layout (one partial result per piece and row, at most two row blocks
+// per branch and KV head), arranged for latency, which is all this kernel costs: one CTA per group
+// (branch, KV head), half a warp per output row; five threads work out where the group's partial
+// results lie, then every thread issues all loads of its row before it uses the first.
+__global__ void __launch_bounds__(512) attn_combine_groups_kernel(const AttnParams p) {
+    extern __shared__ int cum[];                                         // N + 1 ints
+    __shared__ GroupDesc desc;
+    build_branch_tile_prefix(p, cum);
+    const int b = blockIdx.x / p.Hkv, kvh = blockIdx.x - b * p.Hkv;
+    if (threadIdx.x < kMaxPrivBlocks + kMaxPreBlocks)
+        group_describe_entry(p, cum, ceil_div(total_tiles(p, cum), p.grid), b, kvh, threadIdx.x, desc);
+    __syncthreads();
+    merge_group(p, desc, threadIdx.x, blockDim.x);
+}
+
 }  // namespace
 
 cudaError_t launch_attn_combine(const AttnParams& main_params, cudaStream_t st) {
     AttnParams p = main_params;
     p.lens_smem = 0;                     // this kernel's shared memory holds the tile prefix only (N + 1 ints)
+    if (p.copies == 1 && p.copies_pre == 1 && p.n_rb_priv <= kMaxPrivBlocks && p.nr <= 2 * p.rb_rows) {
+        const int threads = min(512, (p.nr * 16 + 31) / 32 * 32);        // 128 registers each: a row's loads are all in flight at once
+        attn_combine_groups_kernel<<<p.N * p.Hkv, threads, (p.N + 1) * sizeof(int), st>>>(p);
+        return cudaGetLastError();
+    }
     const int rows = p.N * p.R * p.Hq;
     attn_combine_kernel<<<ceil_div(rows, kRowsPerBlock), kRowsPerBlock * 32, (p.N + 1) * sizeof(int), st>>>(p);
     return cudaGetLastError();
