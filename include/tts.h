@@ -213,6 +213,30 @@ TTS_API int tts_profile_read(tts_ctx* ctx, float* attn_main_us, float* attn_merg
 TTS_API const char* tts_strerror(int status);
 
 /*
+ * KV-cache bookkeeping either side of the verify step (Section 3.2, sequence-wise parallelism: the
+ * target model scores the last committed token and the gamma drafts of every branch in one pass, so
+ * their keys and values join the branch's cache before the attention, and the cache is cut back to
+ * what was accepted afterwards).
+ *   tts_kv_append: copies the keys and values of the `rows` newest positions of every branch into the
+ *     paged pools, at private tokens branch_lens[b] - rows .. branch_lens[b] - 1 (branch_lens already
+ *     counts them: these are the positions that tts_verify_attn treats as the causal tail).
+ *       k_new, v_new device [n_branches][rows][n_kv_heads][128] bf16 (16-byte aligned), read only
+ *       k_pages, v_pages, block_table, prefix_len, branch_lens as in tts_verify_attn; the pools are written.
+ *     A branch shorter than `rows` or a page index outside [0, num_pages) writes nothing for that
+ *     token and raises TTS_ERR_DEVICE_BOUNDS in the device status (tts_last_status).
+ *   tts_kv_rollback: branch_lens[b] -= gamma - accepted_len[b] (device arrays, i32): the rejected drafts
+ *     leave the cache; the pages stay with the branch.  accepted_len outside [0, gamma] changes nothing
+ *     for that branch and raises TTS_ERR_DEVICE_BOUNDS.
+ * Both are asynchronous on the context's stream; TTS_ERR_INVALID for null or misaligned pointers and
+ * sizes outside the context's limits.
+ */
+TTS_API int tts_kv_append(tts_ctx* ctx, const void* k_new, const void* v_new, void* k_pages, void* v_pages,
+                          const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
+                          int n_branches, int rows);
+TTS_API int tts_kv_rollback(tts_ctx* ctx, int32_t* branch_lens, const int32_t* accepted_len, int n_branches,
+                            int gamma);
+
+/*
  * One whole verify step from HOST buffers (the end-to-end path): for each of n_layers layers,
  * copies that layer's q from pinned host memory, runs tts_verify_attn against that layer's
  * device-resident K/V pools (the KV cache is state that lives in HBM, like the weights) and

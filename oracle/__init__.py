@@ -135,6 +135,44 @@ def majority_vote(answers, weights=None, mode: int = 0):
     return int(w.value), int(v.value), float(s.value)
 
 
+def kv_append(k_pages, v_pages, k_new, v_new, block_table, prefix_len, branch_lens, page_size: int = 16):
+    """KV-cache bookkeeping before the verify step (Section 3.2, speculative decoding: the target model
+    scores the last committed token and the gamma drafts of every branch in one pass, so their keys and
+    values join the cache first).  Token by token, as the definition reads: row i of branch b is private
+    token branch_lens[b] - R + i, i.e. logical token prefix_len + branch_lens[b] - R + i, which lives in
+    page block_table[b][token // page_size] at slot token % page_size.  Pools [num_pages][Hkv][page][D]
+    and new rows [N][R][Hkv][D] as uint16 bf16 bits; returns the two updated pools (copies)."""
+    k = np.array(k_pages, dtype=np.uint16, copy=True)
+    v = np.array(v_pages, dtype=np.uint16, copy=True)
+    k_new = np.asarray(k_new, dtype=np.uint16)
+    v_new = np.asarray(v_new, dtype=np.uint16)
+    n, r = k_new.shape[0], k_new.shape[1]
+    for b in range(n):
+        length = int(branch_lens[b])
+        if length < r:
+            raise ValueError("kv_append: a branch is shorter than the rows appended")
+        for i in range(r):
+            token = prefix_len + length - r + i
+            page = int(block_table[b, token // page_size])
+            slot = token % page_size
+            for h in range(k_new.shape[2]):
+                k[page, h, slot, :] = k_new[b, i, h, :]
+                v[page, h, slot, :] = v_new[b, i, h, :]
+    return k, v
+
+
+def kv_rollback(branch_lens, accepted_len, gamma: int):
+    """After the accept test the gamma - accepted_len rejected drafts of every branch leave the cache
+    (Section 3.2; the resampled or bonus token has no key yet: it is the first row of the next step)."""
+    lens = np.array(branch_lens, dtype=np.int64, copy=True)
+    for b in range(lens.shape[0]):
+        a = int(accepted_len[b])
+        if a < 0 or a > gamma:
+            raise ValueError("kv_rollback: accepted_len outside [0, gamma]")
+        lens[b] = lens[b] - (gamma - a)
+    return lens.astype(np.int32)
+
+
 def greedy_search(acc_table):
     """Algorithm 1 on a dense accuracy table acc[log2 B][gamma].
     Returns (B, gamma, acc, steps, evaluations)."""

@@ -22,7 +22,7 @@ EXPORTED_SYMBOLS = (
     "tts_create", "tts_destroy", "tts_set_stream", "tts_verify_attn", "tts_verify_attn_tree",
     "tts_accept", "tts_majority_vote", "tts_confidence_max", "tts_greedy_search", "tts_last_status",
     "tts_last_cuda_error", "tts_launch_count", "tts_strerror", "tts_verify_step_host",
-    "tts_profile_enable", "tts_profile_read", "tts_verify_attn_noalloc",
+    "tts_profile_enable", "tts_profile_read", "tts_verify_attn_noalloc", "tts_kv_append", "tts_kv_rollback",
 )
 
 
@@ -66,6 +66,8 @@ def load_library() -> ctypes.CDLL:
     lib.tts_verify_attn.argtypes = [vp, vp, vp, vp, vp, c_int, vp, c_int, c_int, c_int, vp]
     lib.tts_verify_attn_tree.argtypes = [vp, vp, vp, vp, vp, c_int, vp, vp, c_int, c_int, vp]
     lib.tts_accept.argtypes = [vp, vp, vp, vp, vp, c_int, c_int, c_int, vp, vp]
+    lib.tts_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, c_int, vp, c_int, c_int]
+    lib.tts_kv_rollback.argtypes = [vp, vp, vp, c_int, c_int]
     lib.tts_majority_vote.argtypes = [POINTER(c_int64), POINTER(c_float), c_int, POINTER(c_int64), POINTER(c_int)]
     lib.tts_confidence_max.argtypes = lib.tts_majority_vote.argtypes
     lib.tts_greedy_search.argtypes = [_TASK_FN, vp, POINTER(c_int), POINTER(c_int), POINTER(c_double), POINTER(c_int)]
@@ -172,6 +174,16 @@ class TtsContext:
         self._check(self._lib.tts_accept(self._h, _ptr(p_target), _ptr(q_draft), _ptr(draft_tokens), _ptr(uniforms),
                                          int(n_branches), int(gamma), int(vocab), _ptr(accepted_len),
                                          _ptr(next_token)), "tts_accept")
+
+    def tts_kv_append(self, k_new, v_new, k_pages, v_pages, block_table, prefix_len: int, branch_lens,
+                      n_branches: int, rows: int):
+        self._check(self._lib.tts_kv_append(self._h, _ptr(k_new), _ptr(v_new), _ptr(k_pages), _ptr(v_pages),
+                                            _ptr(block_table), int(prefix_len), _ptr(branch_lens), int(n_branches),
+                                            int(rows)), "tts_kv_append")
+
+    def tts_kv_rollback(self, branch_lens, accepted_len, n_branches: int, gamma: int):
+        self._check(self._lib.tts_kv_rollback(self._h, _ptr(branch_lens), _ptr(accepted_len), int(n_branches),
+                                              int(gamma)), "tts_kv_rollback")
 
     def tts_last_status(self) -> int:
         st = c_int(0)

@@ -252,6 +252,32 @@ int tts_accept(tts_ctx* ctx, const float* p_target, const float* q_draft, const 
     return TTS_OK;
 }
 
+int tts_kv_append(tts_ctx* ctx, const void* k_new, const void* v_new, void* k_pages, void* v_pages,
+                  const int32_t* block_table, int prefix_len, const int32_t* branch_lens, int n_branches, int rows) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !k_new || !v_new || !k_pages || !v_pages || !block_table || !branch_lens) return TTS_ERR_INVALID;
+    const tts_config& f = c->cfg;
+    if (n_branches < 1 || n_branches > f.max_branches || rows < 1 || rows > f.max_rows_per_branch) return TTS_ERR_INVALID;
+    if (prefix_len < 0 || prefix_len % f.page_size != 0 || prefix_len / f.page_size > f.max_blocks_per_branch)
+        return TTS_ERR_INVALID;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_pages) || !aligned16(v_pages)) return TTS_ERR_INVALID;
+    cudaError_t e = launch_kv_append(k_new, v_new, k_pages, v_pages, block_table, f.max_blocks_per_branch, f.num_pages,
+                                     prefix_len, branch_lens, n_branches, rows, f.n_kv_heads, c->d_status, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->launches += 1;
+    return TTS_OK;
+}
+
+int tts_kv_rollback(tts_ctx* ctx, int32_t* branch_lens, const int32_t* accepted_len, int n_branches, int gamma) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !branch_lens || !accepted_len) return TTS_ERR_INVALID;
+    if (n_branches < 1 || n_branches > c->cfg.max_branches || gamma < 0) return TTS_ERR_INVALID;
+    cudaError_t e = launch_kv_rollback(branch_lens, accepted_len, n_branches, gamma, c->d_status, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->launches += 1;
+    return TTS_OK;
+}
+
 static int vote_impl(const int64_t* answers, const float* weights, int n, int mode, int64_t* winner,
                      int* votes) {
     if (!answers || !winner || n < 1 || (mode == 1 && !weights)) return TTS_ERR_INVALID;
