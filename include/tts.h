@@ -213,6 +213,32 @@ TTS_API int tts_profile_read(tts_ctx* ctx, float* attn_main_us, float* attn_merg
 TTS_API const char* tts_strerror(int status);
 
 /*
+ * Accept test along the paths of a draft tree (tree verification with the tree drafts of the
+ * speculative-decoding models used in Section 4.1; the paper does not spell the rule out, this is the
+ * chain rule of tts_accept applied along every root-to-leaf path).  Per branch, n_nodes tree nodes:
+ *   tree_parents device [n_branches][n_nodes] i32   parent of node i (an index < i), or -1 for a child
+ *                                                   of the last committed token
+ *   draft_tokens device [n_branches][n_nodes] i32   token x_i of node i
+ *   p_target     device [n_branches][n_nodes+1][vocab] fp32   row 0: target distribution after the last
+ *                                                   committed token; row 1 + i: after node i
+ *   q_draft      device [n_branches][n_nodes][vocab] fp32     row i: the draft distribution x_i was drawn from
+ *   uniforms     device [n_branches][n_nodes+1] fp32 in [0,1): u_i for node i, u_{n_nodes} for the final draw
+ * Node i passes iff p(x_i) > 0 and u_i * q_i(x_i) <= p(x_i) (one fp32 multiply), p being row 0 if its
+ * parent is -1 and row 1 + parent otherwise; a node is accepted iff it and all its ancestors pass.  The
+ * leaf whose path holds the most accepted nodes wins (ties: lowest leaf index).
+ *   accepted_len[b] = accepted nodes on the winning path;  last_node[b] = the deepest of them (-1: none);
+ *   next_token[b]   = inverse-CDF draw with u_{n_nodes}, as in tts_accept, from norm(max(0, p - q_k)) for
+ *                     the first node k of the winning path that failed (p: the row of k's parent), or from
+ *                     row 1 + leaf when the whole path was accepted.
+ * A chain (tree_parents[i] = i - 1) gives exactly tts_accept with gamma = n_nodes.  n_nodes <= 64;
+ * vocab % 4 == 0.  Malformed parents or tokens raise TTS_ERR_DEVICE_BOUNDS and count as -1 / token 0.
+ * The rule is not lossless across siblings (a sibling is not re-tested against the residual).
+ */
+TTS_API int tts_accept_tree(tts_ctx* ctx, const float* p_target, const float* q_draft, const int32_t* draft_tokens,
+                            const int32_t* tree_parents, const float* uniforms, int n_branches, int n_nodes,
+                            int vocab, int32_t* accepted_len, int32_t* last_node, int32_t* next_token);
+
+/*
  * KV-cache bookkeeping either side of the verify step (Section 3.2, sequence-wise parallelism: the
  * target model scores the last committed token and the gamma drafts of every branch in one pass, so
  * their keys and values join the branch's cache before the attention, and the cache is cut back to

@@ -2,7 +2,12 @@
 
 Only tests, the smoke check and the benchmark's CPU-baseline / reference legs may import
 this package; the product (paper_2505_19634_b200) never does.  It compiles the C++ file with
-g++ into oracle/_build/ on first use and exposes numpy-in / numpy-out wrappers.
+g++ into oracle/_build/ on first use and exposes numpy-in / numpy-out wrappers; the tree-path accept
+rule and the KV-cache bookkeeping are written here in numpy (token by token, in the order of their
+definitions).
+
+Pins: tests/test_oracle_*.py.  Parity unpinned: one property only, the distribution of the token that
+`accept_tree` emits (its rule is pinned; see its docstring).
 """
 from __future__ import annotations
 
@@ -133,6 +138,96 @@ def majority_vote(answers, weights=None, mode: int = 0):
     if rc != 0:
         raise ValueError("oracle_majority_vote: inconsistent arguments")
     return int(w.value), int(v.value), float(s.value)
+
+
+def accept_tree(p_target, q_draft, draft_tokens, tree_parents, uniforms):
+    """Accept test along the paths of a draft tree: the chain rule of `accept` applied along every
+    root-to-leaf path (tree verification; the paper does not spell the rule out, Section 4.1 only names
+    the drafting models).  Steps, per branch, in this order:
+      1. node i passes iff p(x_i) > 0 and u_i * q_i(x_i) <= p(x_i) with one fp32 multiply, p being row 0
+         of p_target for a child of the last committed token (parent -1) and row 1 + parent otherwise;
+      2. a node is accepted iff it and all its ancestors pass; for every leaf, count the accepted nodes
+         on its path; the leaf with the largest count wins, ties to the lowest leaf index;
+      3. the final draw with u_n: from norm(max(0, p - q_k)) in fp32 (p if that is identically zero) for the
+         first node k of the winning path that failed, p the row of k's parent; or from row 1 + leaf when
+         the whole path was accepted; sums in fp64 in index order, smallest x whose running sum exceeds
+         u_n * Z, else the last x with weight > 0.
+    Returns (accepted_len, last_node, next_token, near_flags) with near_flags as in `accept`.
+    Pinned: a chain reproduces `accept`; brute force over all pass patterns of small trees.  The
+    DISTRIBUTION of the emitted token under this path-selection rule is parity unpinned (the rule is not
+    lossless across siblings, so there is no closed form to test it against)."""
+    P = np.ascontiguousarray(p_target, dtype=np.float32)
+    N, n1, V = P.shape
+    n = n1 - 1
+    Q = np.ascontiguousarray(q_draft, dtype=np.float32).reshape(N, n, V)
+    X = np.ascontiguousarray(draft_tokens, dtype=np.int32).reshape(N, n)
+    PAR = np.ascontiguousarray(tree_parents, dtype=np.int32).reshape(N, n)
+    U = np.ascontiguousarray(uniforms, dtype=np.float32)
+    assert U.shape == (N, n + 1)
+    acc = np.zeros(N, np.int32); last = np.zeros(N, np.int32); nxt = np.zeros(N, np.int32); near = np.zeros(N, np.int32)
+    for b in range(N):
+        flags = 0
+        passes = []
+        for i in range(n):
+            par = int(PAR[b, i])
+            if par < -1 or par >= i:
+                raise ValueError("accept_tree: a parent must be -1 or an earlier node")
+            x = int(X[b, i])
+            p = P[b, par + 1, x]
+            q = Q[b, i, x]
+            uq = np.float32(U[b, i]) * np.float32(q)                       # one fp32 multiply
+            if abs(float(uq) - float(p)) <= 1e-6 * max(float(p), float(q)):
+                flags |= 1
+            passes.append(bool(p > np.float32(0) and uq <= p))
+        children = [[] for _ in range(n)]
+        for i in range(n):
+            if PAR[b, i] >= 0:
+                children[int(PAR[b, i])].append(i)
+        best_leaf, best_count, best_path = -1, -1, []
+        for leaf in range(n):
+            if children[leaf]:
+                continue
+            path = []
+            i = leaf
+            while i >= 0:
+                path.append(i)
+                i = int(PAR[b, i])
+            path.reverse()                                                # root side first
+            count = 0
+            for node in path:
+                if not passes[node]:
+                    break
+                count += 1
+            if count > best_count:
+                best_leaf, best_count, best_path = leaf, count, path
+        if best_leaf < 0:                                                 # no nodes: the bonus token of the committed prefix
+            best_count, best_path = 0, []
+        acc[b] = best_count
+        last[b] = best_path[best_count - 1] if best_count > 0 else -1
+        if best_count < len(best_path):
+            k = best_path[best_count]
+            pk = P[b, int(PAR[b, k]) + 1]
+            r = np.maximum(pk - Q[b, k], np.float32(0)).astype(np.float32)
+            if not (np.cumsum(r.astype(np.float64))[-1] > 0.0):
+                r = pk.copy()
+        else:
+            r = P[b, best_leaf + 1].copy()
+        C = np.cumsum(r.astype(np.float64))                               # sequential fp64 sums in index order
+        Z = float(C[-1])
+        t = float(U[b, n]) * Z
+        over = np.nonzero(C > t)[0]
+        if over.size:
+            chosen = int(over[0])
+            prev = float(C[chosen - 1]) if chosen > 0 else 0.0
+            if abs(float(C[chosen]) - t) <= 1e-9 * Z or (chosen > 0 and abs(t - prev) <= 1e-9 * Z):
+                flags |= 2
+        else:
+            pos = np.nonzero(r > 0)[0]
+            chosen = int(pos[-1]) if pos.size else V - 1
+            flags |= 2
+        nxt[b] = chosen
+        near[b] = flags
+    return acc, last, nxt, near
 
 
 def kv_append(k_pages, v_pages, k_new, v_new, block_table, prefix_len, branch_lens, page_size: int = 16):

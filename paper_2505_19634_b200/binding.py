@@ -22,7 +22,7 @@ EXPORTED_SYMBOLS = (
     "tts_create", "tts_destroy", "tts_set_stream", "tts_verify_attn", "tts_verify_attn_tree",
     "tts_accept", "tts_majority_vote", "tts_confidence_max", "tts_greedy_search", "tts_last_status",
     "tts_last_cuda_error", "tts_launch_count", "tts_strerror", "tts_verify_step_host",
-    "tts_profile_enable", "tts_profile_read", "tts_verify_attn_noalloc", "tts_kv_append", "tts_kv_rollback",
+    "tts_profile_enable", "tts_profile_read", "tts_verify_attn_noalloc", "tts_kv_append", "tts_kv_rollback", "tts_accept_tree",
 )
 
 
@@ -66,6 +66,7 @@ def load_library() -> ctypes.CDLL:
     lib.tts_verify_attn.argtypes = [vp, vp, vp, vp, vp, c_int, vp, c_int, c_int, c_int, vp]
     lib.tts_verify_attn_tree.argtypes = [vp, vp, vp, vp, vp, c_int, vp, vp, c_int, c_int, vp]
     lib.tts_accept.argtypes = [vp, vp, vp, vp, vp, c_int, c_int, c_int, vp, vp]
+    lib.tts_accept_tree.argtypes = [vp, vp, vp, vp, vp, vp, c_int, c_int, c_int, vp, vp, vp]
     lib.tts_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, c_int, vp, c_int, c_int]
     lib.tts_kv_rollback.argtypes = [vp, vp, vp, c_int, c_int]
     lib.tts_majority_vote.argtypes = [POINTER(c_int64), POINTER(c_float), c_int, POINTER(c_int64), POINTER(c_int)]
@@ -174,6 +175,13 @@ class TtsContext:
         self._check(self._lib.tts_accept(self._h, _ptr(p_target), _ptr(q_draft), _ptr(draft_tokens), _ptr(uniforms),
                                          int(n_branches), int(gamma), int(vocab), _ptr(accepted_len),
                                          _ptr(next_token)), "tts_accept")
+
+    def tts_accept_tree(self, p_target, q_draft, draft_tokens, tree_parents, uniforms, n_branches: int, n_nodes: int,
+                        vocab: int, accepted_len, last_node, next_token):
+        self._check(self._lib.tts_accept_tree(self._h, _ptr(p_target), _ptr(q_draft), _ptr(draft_tokens),
+                                              _ptr(tree_parents), _ptr(uniforms), int(n_branches), int(n_nodes),
+                                              int(vocab), _ptr(accepted_len), _ptr(last_node), _ptr(next_token)),
+                    "tts_accept_tree")
 
     def tts_kv_append(self, k_new, v_new, k_pages, v_pages, block_table, prefix_len: int, branch_lens,
                       n_branches: int, rows: int):

@@ -39,43 +39,14 @@ __device__ __forceinline__ float weight(float p, float q, bool residual) {
     return d > 0.f ? d : 0.f;
 }
 
-__global__ void __launch_bounds__(kAccThreads)
-accept_kernel(const float* __restrict__ p_target, const float* __restrict__ q_draft,
-              const int32_t* __restrict__ draft_tokens, const float* __restrict__ uniforms, int gamma,
-              int vocab, int32_t* __restrict__ accepted_len, int32_t* __restrict__ next_token,
-              int32_t* status) {
-    __shared__ double tile_sum[kMaxTiles];
-    __shared__ int s_k, s_last_pos, s_redo;
-
-    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const float* P = p_target + (size_t)b * (gamma + 1) * vocab;
-    const float* Q = q_draft + (size_t)b * gamma * vocab;
-    const float* U = uniforms + (size_t)b * (gamma + 1);
-
-    // ---- 1. accept tests ----
-    if (warp == 0) {
-        int k = gamma;
-        for (int base = 0; base < gamma && k == gamma; base += 32) {
-            const int i = base + lane;
-            bool reject = false;
-            if (i < gamma) {
-                int x = draft_tokens[(size_t)b * gamma + i];
-                if (x < 0 || x >= vocab) { atomicMin(status, (int)TTS_ERR_DEVICE_BOUNDS); x = 0; }
-                const float p = P[(size_t)i * vocab + x];
-                const float q = Q[(size_t)i * vocab + x];
-                const float uq = __fmul_rn(U[i], q);
-                reject = !(p > 0.f && uq <= p);
-            }
-            const unsigned ballot = __ballot_sync(0xffffffffu, reject);
-            if (ballot) k = base + __ffs(ballot) - 1;
-        }
-        if (lane == 0) { s_k = k; s_last_pos = -1; s_redo = 0; accepted_len[b] = k; }
-    }
-    __syncthreads();
-    const int k = s_k;
-    const float* pk = P + (size_t)k * vocab;
-    const float* qk = Q + (size_t)(k < gamma ? k : 0) * vocab;
-    bool residual = k < gamma;
+// Steps 2 and 3 for one branch, by the whole CTA: the draw with u_final from norm(max(0, p - q)) (residual;
+// from p if that is identically zero) or from p.  tile_sum, s_last_pos (-1) and s_redo (0) are shared scratch.
+__device__ __forceinline__ void draw_token(const float* __restrict__ pk, const float* __restrict__ qk, bool residual,
+                                           float u_final, int vocab, double* tile_sum, int* s_last_pos_p, int* s_redo_p,
+                                           int32_t* next_token_out) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int& s_last_pos = *s_last_pos_p;
+    int& s_redo = *s_redo_p;
     const int n_tiles = (vocab + kTileElems - 1) / kTileElems;
 
     double Z = 0.0;
@@ -121,7 +92,7 @@ accept_kernel(const float* __restrict__ p_target, const float* __restrict__ q_dr
 
     // ---- 3b. warp 0: locate the crossing tile, then the token inside it ----
     if (warp == 0) {
-        const double t = (double)U[gamma] * Z;
+        const double t = (double)u_final * Z;
         const int per = (n_tiles + 31) / 32;
         const int j0 = lane * per, j1 = min(n_tiles, (lane + 1) * per);
         double c = 0.0;
@@ -175,9 +146,112 @@ accept_kernel(const float* __restrict__ p_target, const float* __restrict__ q_dr
         }
         if (lane == 0) {
             if (chosen < 0) chosen = s_last_pos >= 0 ? s_last_pos : vocab - 1;   // rounding left no crossing
-            next_token[b] = chosen;
+            *next_token_out = chosen;
         }
     }
+}
+
+__global__ void __launch_bounds__(kAccThreads)
+accept_kernel(const float* __restrict__ p_target, const float* __restrict__ q_draft,
+              const int32_t* __restrict__ draft_tokens, const float* __restrict__ uniforms, int gamma,
+              int vocab, int32_t* __restrict__ accepted_len, int32_t* __restrict__ next_token,
+              int32_t* status) {
+    __shared__ double tile_sum[kMaxTiles];
+    __shared__ int s_k, s_last_pos, s_redo;
+
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float* P = p_target + (size_t)b * (gamma + 1) * vocab;
+    const float* Q = q_draft + (size_t)b * gamma * vocab;
+    const float* U = uniforms + (size_t)b * (gamma + 1);
+
+    // ---- 1. accept tests ----
+    if (warp == 0) {
+        int k = gamma;
+        for (int base = 0; base < gamma && k == gamma; base += 32) {
+            const int i = base + lane;
+            bool reject = false;
+            if (i < gamma) {
+                int x = draft_tokens[(size_t)b * gamma + i];
+                if (x < 0 || x >= vocab) { atomicMin(status, (int)TTS_ERR_DEVICE_BOUNDS); x = 0; }
+                const float p = P[(size_t)i * vocab + x];
+                const float q = Q[(size_t)i * vocab + x];
+                const float uq = __fmul_rn(U[i], q);
+                reject = !(p > 0.f && uq <= p);
+            }
+            const unsigned ballot = __ballot_sync(0xffffffffu, reject);
+            if (ballot) k = base + __ffs(ballot) - 1;
+        }
+        if (lane == 0) { s_k = k; s_last_pos = -1; s_redo = 0; accepted_len[b] = k; }
+    }
+    __syncthreads();
+    const int k = s_k;
+    const float* pk = P + (size_t)k * vocab;
+    const float* qk = Q + (size_t)(k < gamma ? k : 0) * vocab;
+    draw_token(pk, qk, k < gamma, U[gamma], vocab, tile_sum, &s_last_pos, &s_redo, next_token + b);
+}
+
+// The same for a draft tree (n nodes per branch, at most kMaxTreeRows): node i passes iff
+// p_par(i)(x_i) > 0 and u_i q_i(x_i) <= p_par(i)(x_i), p_par(i) being row 0 of p_target for a child of the
+// last committed token and row 1 + parent otherwise; a node is accepted iff it and all its ancestors pass;
+// the leaf whose path holds the most accepted nodes wins (ties: lowest leaf index).  The final draw uses
+// the residual of the first failing node of that path, or row 1 + leaf if the whole path was accepted.
+__global__ void __launch_bounds__(kAccThreads)
+accept_tree_kernel(const float* __restrict__ p_target, const float* __restrict__ q_draft,
+                   const int32_t* __restrict__ draft_tokens, const int32_t* __restrict__ tree_parents,
+                   const float* __restrict__ uniforms, int n, int vocab, int32_t* __restrict__ accepted_len,
+                   int32_t* __restrict__ last_node, int32_t* __restrict__ next_token, int32_t* status) {
+    __shared__ double tile_sum[kMaxTiles];
+    __shared__ int s_last_pos, s_redo, s_row, s_qrow;
+    __shared__ signed char s_pass[kMaxTreeRows], s_par[kMaxTreeRows];
+
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const float* P = p_target + (size_t)b * (n + 1) * vocab;
+    const float* Q = q_draft + (size_t)b * n * vocab;
+    const float* U = uniforms + (size_t)b * (n + 1);
+
+    if (tid < n) {
+        int par = tree_parents[(size_t)b * n + tid];
+        if (par < -1 || par >= tid) { atomicMin(status, (int)TTS_ERR_DEVICE_BOUNDS); par = -1; }
+        int x = draft_tokens[(size_t)b * n + tid];
+        if (x < 0 || x >= vocab) { atomicMin(status, (int)TTS_ERR_DEVICE_BOUNDS); x = 0; }
+        const float p = P[(size_t)(par + 1) * vocab + x];
+        const float q = Q[(size_t)tid * vocab + x];
+        const float uq = __fmul_rn(U[tid], q);
+        s_pass[tid] = (p > 0.f && uq <= p) ? 1 : 0;
+        s_par[tid] = (signed char)par;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        // accepted nodes on the path to i, and whether the whole path to i is accepted (parents come first)
+        signed char alen[kMaxTreeRows], whole[kMaxTreeRows], child[kMaxTreeRows];
+        for (int i = 0; i < n; ++i) child[i] = 0;
+        for (int i = 0; i < n; ++i) {
+            const int par = s_par[i];
+            const bool par_whole = par < 0 || whole[par];
+            whole[i] = par_whole && s_pass[i];
+            alen[i] = (par < 0 ? 0 : alen[par]) + (whole[i] ? 1 : 0);
+            if (par >= 0) child[par] = 1;
+        }
+        int best = -1;
+        for (int i = 0; i < n; ++i)
+            if (!child[i] && (best < 0 || alen[i] > alen[best])) best = i;
+        // walk the winning path up: the deepest accepted node and the failing node right after it
+        int last = -1, fail = -1;
+        for (int i = best; i >= 0; i = s_par[i]) {
+            if (whole[i]) { last = i; break; }
+            fail = i;
+        }
+        accepted_len[b] = best < 0 ? 0 : alen[best];
+        last_node[b] = last;
+        // n == 0: the bonus token of the committed prefix
+        s_row = fail >= 0 ? s_par[fail] + 1 : best + 1;
+        s_qrow = fail;
+        s_last_pos = -1; s_redo = 0;
+    }
+    __syncthreads();
+    const float* pk = P + (size_t)s_row * vocab;
+    const float* qk = Q + (size_t)(s_qrow >= 0 ? s_qrow : 0) * vocab;
+    draw_token(pk, qk, s_qrow >= 0, U[n], vocab, tile_sum, &s_last_pos, &s_redo, next_token + b);
 }
 
 }  // namespace
@@ -188,6 +262,15 @@ cudaError_t launch_accept(const float* p_target, const float* q_draft, const int
                           cudaStream_t st) {
     accept_kernel<<<n_branches, kAccThreads, 0, st>>>(p_target, q_draft, draft_tokens, uniforms,
                                                       gamma, vocab, accepted_len, next_token, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_accept_tree(const float* p_target, const float* q_draft, const int32_t* draft_tokens,
+                               const int32_t* tree_parents, const float* uniforms, int n_branches, int n_nodes, int vocab,
+                               int32_t* accepted_len, int32_t* last_node, int32_t* next_token, int32_t* status,
+                               cudaStream_t st) {
+    accept_tree_kernel<<<n_branches, kAccThreads, 0, st>>>(p_target, q_draft, draft_tokens, tree_parents, uniforms, n_nodes,
+                                                           vocab, accepted_len, last_node, next_token, status);
     return cudaGetLastError();
 }
 

@@ -252,6 +252,22 @@ int tts_accept(tts_ctx* ctx, const float* p_target, const float* q_draft, const 
     return TTS_OK;
 }
 
+int tts_accept_tree(tts_ctx* ctx, const float* p_target, const float* q_draft, const int32_t* draft_tokens,
+                    const int32_t* tree_parents, const float* uniforms, int n_branches, int n_nodes, int vocab,
+                    int32_t* accepted_len, int32_t* last_node, int32_t* next_token) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !p_target || !uniforms || !accepted_len || !last_node || !next_token) return TTS_ERR_INVALID;
+    if (n_nodes < 0 || n_nodes > kMaxTreeRows || n_branches < 1) return TTS_ERR_INVALID;
+    if (n_nodes > 0 && (!q_draft || !draft_tokens || !tree_parents)) return TTS_ERR_INVALID;
+    if (vocab < 4 || vocab % 4 != 0 || vocab > 524288) return TTS_ERR_INVALID;
+    if (!aligned16(p_target) || (q_draft && !aligned16(q_draft))) return TTS_ERR_INVALID;
+    cudaError_t e = launch_accept_tree(p_target, q_draft, draft_tokens, tree_parents, uniforms, n_branches, n_nodes,
+                                       vocab, accepted_len, last_node, next_token, c->d_status, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->launches += 1;
+    return TTS_OK;
+}
+
 int tts_kv_append(tts_ctx* ctx, const void* k_new, const void* v_new, void* k_pages, void* v_pages,
                   const int32_t* block_table, int prefix_len, const int32_t* branch_lens, int n_branches, int rows) {
     Ctx* c = reinterpret_cast<Ctx*>(ctx);

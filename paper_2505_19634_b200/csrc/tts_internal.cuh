@@ -290,6 +290,10 @@ cudaError_t launch_accept(const float* p_target, const float* q_draft, const int
                           const float* uniforms, int n_branches, int gamma, int vocab,
                           int32_t* accepted_len, int32_t* next_token, int32_t* status,
                           cudaStream_t st);
+cudaError_t launch_accept_tree(const float* p_target, const float* q_draft, const int32_t* draft_tokens,
+                               const int32_t* tree_parents, const float* uniforms, int n_branches, int n_nodes, int vocab,
+                               int32_t* accepted_len, int32_t* last_node, int32_t* next_token, int32_t* status,
+                               cudaStream_t st);
 cudaError_t launch_kv_append(const void* k_new, const void* v_new, void* k_pages, void* v_pages,
                              const int32_t* block_table, int max_blocks, int num_pages, int prefix_len,
                              const int32_t* branch_lens, int N, int R, int Hkv, int32_t* status, cudaStream_t st);
