@@ -272,7 +272,11 @@ TTS_API int tts_kv_rollback(tts_ctx* ctx, int32_t* branch_lens, const int32_t* a
  *   k_pools, v_pools   host arrays of n_layers DEVICE pointers
  *   block_table_host, branch_lens_host, p_target_host, q_draft_host, draft_tokens_host,
  *   uniforms_host, accepted_len_host, next_token_host: host copies in the device layouts above.
- * Staging buffers on the device are allocated inside the context on first use.
+ * Staging buffers on the device are allocated inside the context on first use, and so are two
+ * streams of its own on which the copies that need not wait for the kernels run beside them (the
+ * queries of later layers and the accept inputs while the first layers run, the outputs of finished
+ * layers while later ones run); the kernels run on the context's stream.  With pageable host memory
+ * the copies do not overlap anything.
  */
 TTS_API int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const void* const* k_pools,
                          const void* const* v_pools, const int32_t* block_table_host,

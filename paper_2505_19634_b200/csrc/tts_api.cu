@@ -202,6 +202,12 @@ int tts_destroy(tts_ctx* ctx) {
     free_workspace(c);
     cudaFree(c->d_status);
     cudaFree(c->stage);
+    if (c->host_ev) {
+        for (int i = 0; i < kHostEvents; ++i) if (c->host_ev[i]) cudaEventDestroy(c->host_ev[i]);
+        free(c->host_ev);
+    }
+    if (c->h2d_stream) cudaStreamDestroy(c->h2d_stream);
+    if (c->d2h_stream) cudaStreamDestroy(c->d2h_stream);
     if (c->prof_ev) {
         for (int i = 0; i < 3 * kProfMaxCalls; ++i) if (c->prof_ev[i]) cudaEventDestroy(c->prof_ev[i]);
         free(c->prof_ev);
@@ -463,40 +469,84 @@ int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const v
     int32_t* d_al = (int32_t*)base; base += res_b;
     int32_t* d_nt = (int32_t*)base;
 
-    cudaStream_t st = c->stream;
+    // Two more streams carry the copies that need not wait for the kernels: the queries of later layers and
+    // the accept inputs go host-to-device while the first layers run, the outputs of finished layers go back
+    // while later layers run.  Events order them against the context's stream, chunk of layers by chunk.
 #define TTS_CK(x) do { e = (x); if (e != cudaSuccess) return cuda_fail(c, e); } while (0)
+    if (!c->host_ev) {
+        TTS_CK(cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking));
+        TTS_CK(cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking));
+        c->host_ev = static_cast<cudaEvent_t*>(calloc(kHostEvents, sizeof(cudaEvent_t)));
+        if (!c->host_ev) return TTS_ERR_INVALID;
+        for (int i = 0; i < kHostEvents; ++i) TTS_CK(cudaEventCreateWithFlags(&c->host_ev[i], cudaEventDisableTiming));
+    }
+    cudaStream_t st = c->stream, up_st = c->h2d_stream, down_st = c->d2h_stream;
+    cudaEvent_t* ev_q = c->host_ev;                         // queries of chunk i are on the device
+    cudaEvent_t* ev_o = c->host_ev + kHostChunks;           // outputs of chunk i are computed
+    cudaEvent_t ev_start = c->host_ev[2 * kHostChunks], ev_acc = c->host_ev[2 * kHostChunks + 1];
+    const int per_chunk = (n_layers + kHostChunks - 1) / kHostChunks < 4 ? (n_layers < 4 ? n_layers : 4)
+                                                                         : (n_layers + kHostChunks - 1) / kHostChunks;
+    const int n_chunks = (n_layers + per_chunk - 1) / per_chunk;
+    // the staging buffers may still be read by work queued on the context's stream before this call
+    TTS_CK(cudaEventRecord(ev_start, st));
+    TTS_CK(cudaStreamWaitEvent(up_st, ev_start, 0));
+    TTS_CK(cudaStreamWaitEvent(down_st, ev_start, 0));
     TTS_CK(cudaMemcpyAsync(d_bt, block_table_host, (size_t)n_branches * f.max_blocks_per_branch * 4, cudaMemcpyHostToDevice, st));
     TTS_CK(cudaMemcpyAsync(d_bl, branch_lens_host, (size_t)n_branches * 4, cudaMemcpyHostToDevice, st));
-    // all layers' queries in one copy (they are contiguous on the host)
-    if (up(q_layer) == q_layer) {
-        TTS_CK(cudaMemcpyAsync(d_q, q_host, q_layer * n_layers, cudaMemcpyHostToDevice, st));
-    } else {
-        for (int l = 0; l < n_layers; ++l)
-            TTS_CK(cudaMemcpyAsync(d_q + up(q_layer) * l, (const char*)q_host + q_layer * l, q_layer, cudaMemcpyHostToDevice, st));
+    auto copy_q = [&](int l0, int l1, cudaStream_t s2) -> cudaError_t {
+        if (up(q_layer) == q_layer)                         // contiguous on both sides: one copy
+            return cudaMemcpyAsync(d_q + q_layer * l0, (const char*)q_host + q_layer * l0, q_layer * (l1 - l0), cudaMemcpyHostToDevice, s2);
+        for (int l = l0; l < l1; ++l) {
+            cudaError_t e2 = cudaMemcpyAsync(d_q + up(q_layer) * l, (const char*)q_host + q_layer * l, q_layer, cudaMemcpyHostToDevice, s2);
+            if (e2 != cudaSuccess) return e2;
+        }
+        return cudaSuccess;
+    };
+    auto copy_o = [&](int l0, int l1, cudaStream_t s2) -> cudaError_t {
+        if (up(o_layer) == o_layer)
+            return cudaMemcpyAsync((char*)out_host + o_layer * l0, d_o + o_layer * l0, o_layer * (l1 - l0), cudaMemcpyDeviceToHost, s2);
+        for (int l = l0; l < l1; ++l) {
+            cudaError_t e2 = cudaMemcpyAsync((char*)out_host + o_layer * l, d_o + up(o_layer) * l, o_layer, cudaMemcpyDeviceToHost, s2);
+            if (e2 != cudaSuccess) return e2;
+        }
+        return cudaSuccess;
+    };
+    // host-to-device: the first chunk of queries on the context's stream, the rest and the accept inputs beside it
+    TTS_CK(copy_q(0, per_chunk < n_layers ? per_chunk : n_layers, st));
+    for (int ch = 1; ch < n_chunks; ++ch) {
+        const int l0 = ch * per_chunk, l1 = l0 + per_chunk < n_layers ? l0 + per_chunk : n_layers;
+        TTS_CK(copy_q(l0, l1, up_st));
+        TTS_CK(cudaEventRecord(ev_q[ch], up_st));
     }
-    for (int l = 0; l < n_layers; ++l) {
-        int rc = tts_verify_attn(ctx, d_q + up(q_layer) * l, k_pools[l], v_pools[l], d_bt, prefix_len, d_bl,
-                                 n_branches, gamma, TTS_MASK_CAUSAL, d_o + up(o_layer) * l);
-        if (rc != TTS_OK) return rc;
-    }
-    if (up(o_layer) == o_layer) {
-        TTS_CK(cudaMemcpyAsync(out_host, d_o, o_layer * n_layers, cudaMemcpyDeviceToHost, st));
-    } else {
-        for (int l = 0; l < n_layers; ++l)
-            TTS_CK(cudaMemcpyAsync((char*)out_host + o_layer * l, d_o + up(o_layer) * l, o_layer, cudaMemcpyDeviceToHost, st));
-    }
-    TTS_CK(cudaMemcpyAsync(d_pt, p_target_host, (size_t)n_branches * (gamma + 1) * vocab * 4, cudaMemcpyHostToDevice, st));
+    TTS_CK(cudaMemcpyAsync(d_pt, p_target_host, (size_t)n_branches * (gamma + 1) * vocab * 4, cudaMemcpyHostToDevice, up_st));
     if (gamma > 0) {
-        TTS_CK(cudaMemcpyAsync(d_qd, q_draft_host, (size_t)n_branches * gamma * vocab * 4, cudaMemcpyHostToDevice, st));
-        TTS_CK(cudaMemcpyAsync(d_dt, draft_tokens_host, (size_t)n_branches * gamma * 4, cudaMemcpyHostToDevice, st));
+        TTS_CK(cudaMemcpyAsync(d_qd, q_draft_host, (size_t)n_branches * gamma * vocab * 4, cudaMemcpyHostToDevice, up_st));
+        TTS_CK(cudaMemcpyAsync(d_dt, draft_tokens_host, (size_t)n_branches * gamma * 4, cudaMemcpyHostToDevice, up_st));
     }
-    TTS_CK(cudaMemcpyAsync(d_un, uniforms_host, (size_t)n_branches * (gamma + 1) * 4, cudaMemcpyHostToDevice, st));
+    TTS_CK(cudaMemcpyAsync(d_un, uniforms_host, (size_t)n_branches * (gamma + 1) * 4, cudaMemcpyHostToDevice, up_st));
+    TTS_CK(cudaEventRecord(ev_acc, up_st));
+    // the layers, chunk by chunk; every finished chunk's outputs go back beside the next chunk's kernels
+    for (int ch = 0; ch < n_chunks; ++ch) {
+        const int l0 = ch * per_chunk, l1 = l0 + per_chunk < n_layers ? l0 + per_chunk : n_layers;
+        if (ch > 0) TTS_CK(cudaStreamWaitEvent(st, ev_q[ch], 0));
+        for (int l = l0; l < l1; ++l) {
+            int rc = tts_verify_attn(ctx, d_q + up(q_layer) * l, k_pools[l], v_pools[l], d_bt, prefix_len, d_bl,
+                                     n_branches, gamma, TTS_MASK_CAUSAL, d_o + up(o_layer) * l);
+            if (rc != TTS_OK) return rc;
+        }
+        TTS_CK(cudaEventRecord(ev_o[ch], st));
+        TTS_CK(cudaStreamWaitEvent(down_st, ev_o[ch], 0));
+        TTS_CK(copy_o(l0, l1, down_st));
+    }
+    TTS_CK(cudaStreamWaitEvent(st, ev_acc, 0));
     int rc = tts_accept(ctx, d_pt, gamma > 0 ? d_qd : nullptr, gamma > 0 ? d_dt : nullptr, d_un, n_branches, gamma,
                         vocab, d_al, d_nt);
     if (rc != TTS_OK) return rc;
     TTS_CK(cudaMemcpyAsync(accepted_len_host, d_al, (size_t)n_branches * 4, cudaMemcpyDeviceToHost, st));
     TTS_CK(cudaMemcpyAsync(next_token_host, d_nt, (size_t)n_branches * 4, cudaMemcpyDeviceToHost, st));
     TTS_CK(cudaStreamSynchronize(st));
+    TTS_CK(cudaStreamSynchronize(down_st));
+    TTS_CK(cudaStreamSynchronize(up_st));
 #undef TTS_CK
     return TTS_OK;
 }

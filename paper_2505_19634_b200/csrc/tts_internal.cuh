@@ -276,12 +276,16 @@ struct Ctx {
     size_t pre_rows, priv_rows;       // allocated partial rows (each 128 fp32 + one float2)
     // staging for the host entry point
     void* stage; size_t stage_bytes;
+    cudaStream_t h2d_stream, d2h_stream;   // copies of the host entry point that overlap the kernels (created on first use)
+    cudaEvent_t* host_ev;                  // kHostEvents events ordering them against the context's stream
     void* tmap_cache;                  // opaque: tensor maps keyed by pool pointer
     // profiling aid
     int profiling, prof_n;
     cudaEvent_t* prof_ev;              // 3 events per recorded call
 };
 constexpr int kProfMaxCalls = 4096;
+constexpr int kHostChunks = 16;       // the host entry point moves queries and outputs in at most this many chunks of layers
+constexpr int kHostEvents = 2 * kHostChunks + 2;
 
 // kernel launchers (each returns the cudaError_t of its launch)
 cudaError_t launch_attn_simt(const AttnParams& p, cudaStream_t st);
