@@ -106,13 +106,13 @@ class AttnShape:
 
 
 CONFIGS: Dict[str, AttnShape] = {
-    # BASELINE configs[0]
+    # the small case (the oracle finishes it in seconds)
     "tiny": AttnShape("tiny", n_q_heads=8, n_kv_heads=2, prefix_len=256, n_branches=4, gamma=3,
                       private_len=256, permute_pages=False, vocab=1024, logit_sigma=2.0),
-    # BASELINE configs[1]
+    # Qwen2.5-3B-shaped layer
     "3b": AttnShape("3b", n_q_heads=16, n_kv_heads=2, prefix_len=512, n_branches=8, gamma=4,
                     private_len=2048, vocab=151936, logit_sigma=3.0),
-    # BASELINE configs[2]
+    # Qwen2.5-32B-shaped layer, 64 of them per step: the benchmark's workload
     "32b": AttnShape("32b", n_q_heads=40, n_kv_heads=8, prefix_len=512, n_branches=16, gamma=3,
                      private_len=4096, n_layers=64, vocab=152064, logit_sigma=3.0),
 }
@@ -122,7 +122,7 @@ SWEEP_GAMMAS = (1, 3, 5)
 
 
 def sweep_shape(n_branches: int, gamma: int, seed: int, lo: int = 1024, hi: int = 8192) -> AttnShape:
-    """BASELINE configs[3]: 32B layer shape, ragged private lengths U{lo..hi},
+    """The branch / gamma sweep: 32B layer shape, ragged private lengths U{lo..hi},
     shared prefix 16*U{16..64}, random page permutation."""
     rng = _rng(seed, 911)
     lens = rng.integers(lo, hi + 1, size=n_branches)
@@ -281,7 +281,7 @@ def make_accept_case(n_branches: int, gamma: int, vocab: int, sigma: float, seed
                      draft_noise: Optional[float] = None) -> AcceptCase:
     """Target and draft logits ~ N(0, sigma) (sigma = standard deviation).
 
-    draft_noise=None: independent target and draft logits (BASELINE recipe).
+    draft_noise=None: independent target and draft logits (the default recipe).
     draft_noise=tau: draft logits = target logits + N(0, tau), which gives the high
     acceptance rates (0.7..0.9) the paper reports for its model pairs (Appendix A.1).
     Draft tokens are drawn from q_draft."""
