@@ -109,10 +109,16 @@ __global__ void __launch_bounds__(kRowsPerBlock * 32) attn_combine_kernel(const 
 __global__ void __launch_bounds__(512) attn_combine_groups_kernel(const AttnParams p) {
     extern __shared__ int cum[];                                         // N + 1 ints
     __shared__ GroupDesc desc;
-    build_branch_tile_prefix(p, cum);
-    const int b = blockIdx.x / p.Hkv, kvh = blockIdx.x - b * p.Hkv;
-    if (threadIdx.x < kMaxPrivBlocks + kMaxPreBlocks)
-        group_describe_entry(p, cum, ceil_div(total_tiles(p, cum), p.grid), b, kvh, threadIdx.x, desc);
+    static_assert(sizeof(GroupDesc) % sizeof(int) == 0, "GroupDesc is copied word by word");
+    if (p.group_desc) {                                                  // the main kernel has worked it out
+        if (threadIdx.x < sizeof(GroupDesc) / sizeof(int))
+            reinterpret_cast<int*>(&desc)[threadIdx.x] = reinterpret_cast<const int*>(static_cast<const GroupDesc*>(p.group_desc) + blockIdx.x)[threadIdx.x];
+    } else {
+        build_branch_tile_prefix(p, cum);
+        const int b = blockIdx.x / p.Hkv, kvh = blockIdx.x - b * p.Hkv;
+        if (threadIdx.x < kMaxPrivBlocks + kMaxPreBlocks)
+            group_describe_entry(p, cum, ceil_div(total_tiles(p, cum), p.grid), b, kvh, threadIdx.x, desc);
+    }
     __syncthreads();
     merge_group(p, desc, threadIdx.x, blockDim.x);
 }

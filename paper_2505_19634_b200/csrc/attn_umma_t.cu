@@ -45,6 +45,7 @@
 
 #include <type_traits>
 
+#include "attn_merge.cuh"
 #include "tts_internal.cuh"
 #include "umma_ptx.cuh"
 
@@ -240,6 +241,12 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     SegInfo seg0;
     if (has_work) seg0 = segment_in_group(p, cum, group0, g_begin);
 
+    // Where the partial results of every group (branch, KV head) lie, for the merge kernel: a function of the
+    // schedule alone; the first epilogue warp, idle until the first piece ends, writes it for the groups that
+    // fall to this CTA (five lanes per group, one per entry).
+    if (warp == kEpilogueWarp && p.group_desc && lane < kMaxPrivBlocks + kMaxPreBlocks)
+        for (int grp = blockIdx.x; grp < p.N * p.Hkv; grp += gridDim.x)
+            group_describe_entry(p, cum, tpc, grp / p.Hkv, grp % p.Hkv, lane, static_cast<GroupDesc*>(p.group_desc)[grp]);
     if (!has_work) {
         // nothing to do for this CTA
     } else if (warp == kProducerWarp || warp == kProducerWarp + 1) {

@@ -44,6 +44,7 @@ Plan make_plan(const Ctx* c, int nr, int n_branches) {
 
 void free_workspace(Ctx* c) {
     cudaFree(c->part_o_pre); cudaFree(c->part_ml_pre); cudaFree(c->part_o_priv); cudaFree(c->part_ml_priv);
+    cudaFree(c->group_desc); c->group_desc = nullptr;
     c->part_o_pre = c->part_o_priv = nullptr; c->part_ml_pre = c->part_ml_priv = nullptr;
     c->pre_rows = c->priv_rows = 0;
 }
@@ -82,7 +83,7 @@ cudaError_t alloc_workspace(Ctx* c) {
     if ((e = cudaMalloc(&c->part_o_priv, priv * kHeadDim * sizeof(float))) != cudaSuccess) return e;
     if ((e = cudaMalloc(&c->part_ml_priv, priv * sizeof(float2))) != cudaSuccess) return e;
     c->pre_rows = pre; c->priv_rows = priv;
-    return cudaSuccess;
+    return cudaMalloc(&c->group_desc, (size_t)f.max_branches * f.n_kv_heads * 64);   // a GroupDesc is 48 bytes
 }
 
 int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
@@ -122,6 +123,8 @@ int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
     p.part_o_pre = c->part_o_pre; p.part_ml_pre = c->part_ml_pre;
     p.part_o_priv = c->part_o_priv; p.part_ml_priv = c->part_ml_priv;
     p.status = c->d_status;
+    // the token-major kernel tells the merge kernel where every group's partial results lie
+    p.group_desc = pl.impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR ? c->group_desc : nullptr;
     p.N = n_branches; p.R = rows; p.Hq = f.n_q_heads; p.Hkv = f.n_kv_heads; p.G = G; p.nr = nr;
     p.P = prefix_len; p.max_blocks = f.max_blocks_per_branch; p.num_pages = f.num_pages;
     p.rb_rows = pl.rb_rows;

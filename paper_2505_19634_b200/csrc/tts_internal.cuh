@@ -43,6 +43,7 @@ struct AttnParams {
     float* part_o_priv;   // [N*Hkv*n_rb_priv + grid][priv_stride][128]
     float2* part_ml_priv;
     int32_t* status;      // device status word
+    void* group_desc;     // [N*Hkv] GroupDesc (attn_merge.cuh) written by the main kernel for the merge kernel, or null
     int N, R, Hq, Hkv, G, nr;      // nr = R*G rows per (branch, kv head)
     int P;                          // prefix tokens
     int max_blocks, num_pages;
@@ -274,6 +275,7 @@ struct Ctx {
     // split-KV workspace
     float* part_o_pre; float2* part_ml_pre; float* part_o_priv; float2* part_ml_priv;
     size_t pre_rows, priv_rows;       // allocated partial rows (each 128 fp32 + one float2)
+    void* group_desc;                 // one merge descriptor per (branch, KV head)
     // staging for the host entry point
     void* stage; size_t stage_bytes;
     cudaStream_t h2d_stream, d2h_stream;   // copies of the host entry point that overlap the kernels (created on first use)
