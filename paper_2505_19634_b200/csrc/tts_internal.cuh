@@ -224,8 +224,9 @@ __device__ inline SegInfo next_segment(const AttnParams& p, const int* cum, cons
 
 // First tile of prefix segment s: it follows the first group idx with pre_before(idx + 1) > s.
 __device__ inline int prefix_segment_tile_begin(const AttnParams& p, const int* cum, int s) {
-    const long long n_groups = (long long)p.N * p.Hkv;
-    const int idx = (int)(((long long)(s + 1) * n_groups + p.n_pre - 1) / p.n_pre) - 1;
+    // (s + 1) * groups + n_pre - 1 <= groups * n_pre + n_pre < 2^32: the host rejects groups * n_pre >= 2^31
+    const unsigned int n_groups = (unsigned int)(p.N * p.Hkv);
+    const int idx = (int)(((unsigned int)(s + 1) * n_groups + (unsigned int)p.n_pre - 1u) / (unsigned int)p.n_pre) - 1;
     const int b = idx / p.Hkv;
     const int tb = cum[b + 1] - cum[b];
     return group_tile_begin(p, cum, idx) + p.n_rb_priv * tb + (s - pre_before(p, idx)) * p.tiles_pre;
