@@ -307,7 +307,7 @@ def run_ours(args, shape):
         layer_bytes = shape.unique_kv_bytes()
         # DRAM read + write bytes of one launch of the dominant kernel, from the ncu capture summarised in
         # profiles/attn_umma_t_kernel_32b_2layers.md (valid for the 32b workload and this kernel version only)
-        traffic = 276.9e6 if shape.name == "32b" else None
+        traffic = 276.4e6 if shape.name == "32b" else None
         roof = {"bound": "hbm", "achieved": None, "peak": peak, "unit": "GB/s", "frac": None, "traffic": traffic,
                 "peak_kind": f"of {peak_kind}", "kernel": "attn_umma_t_kernel (token-major tcgen05 attention, one layer per launch)"}
         if main_us:
