@@ -4,10 +4,12 @@
  * The verify step of batched speculative decoding for test-time scaling: the target model
  * scores N concurrent branches of one question (branch-wise parallelism, Section 3.2), each
  * carrying gamma draft tokens plus one bonus position (sequence-wise parallelism, Section 3.2;
- * "verify them in parallel while ensuring a lossless acceleration", Section 2).  The library
- * covers the two parts of that step that are not weight GEMMs:
- *   (1) GQA attention of the N*(gamma+1) query positions over a paged KV cache ("KV caches are
- *       loaded from HBM", Section 3.1) whose prompt prefix is shared by all branches, and
+ * the target checks all gamma drafts in one pass and the output distribution stays the
+ * target's own, Section 2).  The library covers the two parts of that step that are not weight
+ * GEMMs:
+ *   (1) GQA attention of the N*(gamma+1) query positions over a paged KV cache (the cache is
+ *       streamed from HBM at every step, Section 3.1) whose prompt prefix is shared by all
+ *       branches, and
  *   (2) the speculative-sampling accept / residual-resample pass,
  * plus the host-side answer aggregation (majority voting, Section 3.2; confidence-weighted
  * variants, Section 4.6) and the greedy (B, gamma) search (Algorithm 1).
@@ -72,8 +74,11 @@ typedef struct {
     int32_t out_dtype;             /* TTS_OUT_BF16 (round to nearest even) or TTS_OUT_FP32 */
     int32_t attn_impl;             /* TTS_ATTN_* */
     float   softmax_scale;         /* 0 => 1/sqrt(head_dim) */
-    int32_t debug_bounds;          /* != 0: kernels range-check page ids and lengths, report through
-                                      tts_last_status instead of reading out of range */
+    int32_t debug_bounds;          /* != 0: the kernels range-check block indices and page ids and report
+                                      through tts_last_status instead of reading out of range */
+    int32_t max_ctas;              /* 0: the attention kernels size their grids from the SM count; > 0: upper
+                                      bound on the CTAs of the main attention kernel.  It changes how the KV
+                                      tokens are split between CTAs, not what is computed (tuning / tests) */
 } tts_config;
 
 /* Creates a context on the CURRENT CUDA device and allocates its workspace there (split-KV
@@ -104,8 +109,12 @@ TTS_API int tts_set_stream(tts_ctx* ctx, void* cuda_stream);
  *                        gamma+1 in-flight positions, whose K/V are already in the pages;
  *                        precondition branch_lens[b] >= gamma+1
  *   mask_kind    TTS_MASK_CAUSAL (TTS_MASK_TREE: use tts_verify_attn_tree)
- * Errors: INVALID / UNSUPPORTED from host-side checks, CUDA on launch failure.  Device-side
- * preconditions are checked only when cfg.debug_bounds != 0.
+ * Errors: INVALID / UNSUPPORTED from host-side checks, CUDA on launch failure.  What lives on the
+ * device cannot be checked by the host: branch_lens[b] >= gamma+1, prefix_len + branch_lens[b] <=
+ * 16 * max_blocks_per_branch, and page ids in [0, num_pages) are preconditions.  With
+ * cfg.debug_bounds != 0 the kernels test the last two: a block index past the table row or a page id
+ * outside the pool raises TTS_ERR_DEVICE_BOUNDS (tts_last_status) and page 0 is read in its place;
+ * without it such a call reads out of range.
  */
 TTS_API int tts_verify_attn(tts_ctx* ctx, const void* q, const void* k_pages, const void* v_pages,
                     const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
@@ -145,7 +154,11 @@ TTS_API int tts_verify_attn_tree(tts_ctx* ctx, const void* q, const void* k_page
  *   - all calls share the one array, which keeps the previous call's contents (the status word in it
  *     is cleared on the stream at every call; nothing else needs clearing); two calls whose kernels
  *     may overlap on the GPU (different streams, no dependency) race on it - serialise them;
- *   - device-side preconditions (page ids in range, branch_lens >= gamma+1) are not checked.
+ *   - device-side preconditions (page ids in range, branch_lens >= gamma+1, prefix_len + branch_lens
+ *     within the table row) are not checked, and the status word that the kernels keep in the array
+ *     has no accessor: a caller cannot read it;
+ *   - the array's address is looked up once per device and kept: after cudaDeviceReset on that device
+ *     the kept address is stale and this entry point must not be called again in the process.
  */
 TTS_API int tts_verify_attn_noalloc(const void* q, const void* k_pages, const void* v_pages,
                             const int32_t* block_table, int max_blocks_per_branch, int prefix_len,
@@ -175,7 +188,7 @@ TTS_API int tts_accept(tts_ctx* ctx, const float* p_target, const float* q_draft
  *     with the largest weight sum ("vote" aggregation of Section 4.6); ties go to the answer whose
  *     first occurrence has the lowest branch index.  votes = branches that gave the winner.
  *   tts_confidence_max: answer of the single branch with the largest weight ("max" aggregation of
- *     Section 4.6; ties: lowest branch index).
+ *     Section 4.6; ties: lowest branch index); weights must not be NULL.
  */
 TTS_API int tts_majority_vote(const int64_t* answers, const float* weights, int n, int64_t* winner,
                       int* votes);
@@ -183,15 +196,32 @@ TTS_API int tts_confidence_max(const int64_t* answers, const float* weights, int
                        int* votes);
 
 /*
- * Greedy search for the latency-optimal (B, gamma) (Algorithm 1).  Host only.  tts_task is called
- * as tts_task(B, gamma, user) and returns the accuracy reached within the caller's latency budget;
- * a negative return marks the point as unavailable (outside the caller's range).  Starts at
- * (1, 0); each step evaluates (2B, gamma) and (B, gamma+1), moves to the better one (branch-wise
- * on ties) if it improves, stops otherwise.  steps = loop iterations.
+ * Search for the latency-optimal configuration (B, gamma) (Section 3.3, Algorithm 1; compared with
+ * the exhaustive grid in Section 4.5).  Host only.  The configurations form a lattice: B = 1, 2, 4, ..
+ * up to limits->max_branches, gamma = 0 .. limits->max_gamma.  tts_task(B, gamma, user) returns the
+ * accuracy the caller reaches with that configuration inside its latency budget; a negative return
+ * marks the point as unavailable.  limits == NULL means B <= 64, gamma <= 7 (the ranges of Section
+ * 4.5) and at most 64 steps.
+ *   tts_greedy_search: hill climbing from (1, 0).  Each step scores the two neighbours (2B, gamma) and
+ *     (B, gamma+1) that lie inside the lattice, and moves to the better one if it beats the current
+ *     point (equal neighbours: more branches); it stops at the first step that brings no improvement,
+ *     or after limits->max_steps steps.  steps = steps taken including the last, unsuccessful one;
+ *     evaluations = calls of tts_task.
+ *   tts_grid_search: scores every lattice point, (log2 max_branches + 1) * (max_gamma + 1) calls, and
+ *     returns the best (equal optima: the first in (B, gamma) order).
+ * best_acc, steps and evaluations may be NULL.  TTS_ERR_INVALID for null callbacks or limits outside
+ * 1 <= max_branches <= 2^20, 0 <= max_gamma <= 4096.
  */
 typedef double (*tts_task_fn)(int n_branches, int gamma, void* user);
-TTS_API int tts_greedy_search(tts_task_fn tts_task, void* user, int* best_branches, int* best_gamma,
-                      double* best_acc, int* steps);
+typedef struct {
+    int32_t max_branches;   /* largest B tried (the lattice holds the powers of two up to it) */
+    int32_t max_gamma;      /* largest draft length tried */
+    int32_t max_steps;      /* greedy search: upper bound on steps; <= 0 means 64 */
+} tts_search_limits;
+TTS_API int tts_greedy_search(tts_task_fn tts_task, void* user, const tts_search_limits* limits,
+                      int* best_branches, int* best_gamma, double* best_acc, int* steps, int* evaluations);
+TTS_API int tts_grid_search(tts_task_fn tts_task, void* user, const tts_search_limits* limits,
+                    int* best_branches, int* best_gamma, double* best_acc, int* evaluations);
 
 /* Synchronises the stream and reads the device status word: TTS_OK, TTS_ERR_DEVICE_BOUNDS or
  * TTS_ERR_DEVICE_TIMEOUT, written to *device_status; clears it.  Host pointers. */

@@ -280,3 +280,17 @@ def greedy_search(acc_table):
     if rc != 0:
         raise ValueError("oracle_greedy_search: inconsistent arguments")
     return 1 << lb.value, g.value, a.value, st.value, ev.value
+
+
+def grid_search(acc_table):
+    """The exhaustive baseline of Section 3.3 / Section 4.5: every configuration of the table
+    acc[log2 B][gamma] is evaluated once and the most accurate one is kept (equal optima: the first
+    in (B, gamma) order).  Returns (B, gamma, acc, evaluations)."""
+    t = np.asarray(acc_table, dtype=np.float64)
+    best, evaluations = None, 0
+    for lb in range(t.shape[0]):
+        for g in range(t.shape[1]):
+            evaluations += 1
+            if best is None or t[lb, g] > best[2]:
+                best = (1 << lb, g, float(t[lb, g]))
+    return best[0], best[1], best[2], evaluations

@@ -20,7 +20,7 @@ ATTN_AUTO, ATTN_SIMT, ATTN_TCGEN05, ATTN_TCGEN05_TOKEN_MAJOR, ATTN_TCGEN05_ROW_M
 
 EXPORTED_SYMBOLS = (
     "tts_create", "tts_destroy", "tts_set_stream", "tts_verify_attn", "tts_verify_attn_tree",
-    "tts_accept", "tts_majority_vote", "tts_confidence_max", "tts_greedy_search", "tts_last_status",
+    "tts_accept", "tts_majority_vote", "tts_confidence_max", "tts_greedy_search", "tts_grid_search", "tts_last_status",
     "tts_last_cuda_error", "tts_launch_count", "tts_strerror", "tts_verify_step_host",
     "tts_profile_enable", "tts_profile_read", "tts_verify_attn_noalloc", "tts_kv_append", "tts_kv_rollback", "tts_accept_tree",
 )
@@ -38,7 +38,12 @@ class TtsConfig(ctypes.Structure):
     _fields_ = [("n_q_heads", c_int32), ("n_kv_heads", c_int32), ("head_dim", c_int32),
                 ("page_size", c_int32), ("max_branches", c_int32), ("max_rows_per_branch", c_int32),
                 ("max_blocks_per_branch", c_int32), ("num_pages", c_int32), ("out_dtype", c_int32),
-                ("attn_impl", c_int32), ("softmax_scale", c_float), ("debug_bounds", c_int32)]
+                ("attn_impl", c_int32), ("softmax_scale", c_float), ("debug_bounds", c_int32),
+                ("max_ctas", c_int32)]
+
+
+class TtsSearchLimits(ctypes.Structure):
+    _fields_ = [("max_branches", c_int32), ("max_gamma", c_int32), ("max_steps", c_int32)]
 
 
 _TASK_FN = ctypes.CFUNCTYPE(c_double, c_int, c_int, c_void_p)
@@ -71,7 +76,10 @@ def load_library() -> ctypes.CDLL:
     lib.tts_kv_rollback.argtypes = [vp, vp, vp, c_int, c_int]
     lib.tts_majority_vote.argtypes = [POINTER(c_int64), POINTER(c_float), c_int, POINTER(c_int64), POINTER(c_int)]
     lib.tts_confidence_max.argtypes = lib.tts_majority_vote.argtypes
-    lib.tts_greedy_search.argtypes = [_TASK_FN, vp, POINTER(c_int), POINTER(c_int), POINTER(c_double), POINTER(c_int)]
+    lib.tts_greedy_search.argtypes = [_TASK_FN, vp, POINTER(TtsSearchLimits), POINTER(c_int), POINTER(c_int),
+                                      POINTER(c_double), POINTER(c_int), POINTER(c_int)]
+    lib.tts_grid_search.argtypes = [_TASK_FN, vp, POINTER(TtsSearchLimits), POINTER(c_int), POINTER(c_int),
+                                    POINTER(c_double), POINTER(c_int)]
     lib.tts_last_status.argtypes = [vp, POINTER(c_int)]
     lib.tts_last_cuda_error.argtypes = [vp]
     lib.tts_launch_count.argtypes = [vp]
@@ -117,11 +125,11 @@ class TtsContext:
     def __init__(self, n_q_heads: int, n_kv_heads: int, max_branches: int, max_rows_per_branch: int,
                  max_blocks_per_branch: int, num_pages: int, out_dtype: int = OUT_BF16,
                  attn_impl: int = ATTN_AUTO, softmax_scale: float = 0.0, debug_bounds: bool = False,
-                 head_dim: int = 128, page_size: int = 16, stream=None):
+                 head_dim: int = 128, page_size: int = 16, stream=None, max_ctas: int = 0):
         self._lib = load_library()
         self.cfg = TtsConfig(n_q_heads, n_kv_heads, head_dim, page_size, max_branches, max_rows_per_branch,
                              max_blocks_per_branch, num_pages, out_dtype, attn_impl, softmax_scale,
-                             1 if debug_bounds else 0)
+                             1 if debug_bounds else 0, int(max_ctas))
         self._h = c_void_p(0)
         rc = self._lib.tts_create(byref(self.cfg), byref(self._h))
         if rc != 0:
@@ -262,13 +270,33 @@ def tts_confidence_max(answers, weights):
     return _vote("tts_confidence_max", answers, weights)
 
 
-def tts_greedy_search(tts_task):
-    """Algorithm 1 over a Python callable tts_task(B, gamma) -> accuracy (negative = unavailable).
-    Returns (B, gamma, accuracy, steps)."""
+def _limits(max_branches, max_gamma, max_steps):
+    if max_branches is None and max_gamma is None and max_steps is None:
+        return None
+    return byref(TtsSearchLimits(64 if max_branches is None else int(max_branches),
+                                 7 if max_gamma is None else int(max_gamma), int(max_steps or 0)))
+
+
+def tts_greedy_search(tts_task, max_branches=None, max_gamma=None, max_steps=None):
+    """Greedy (B, gamma) search over a Python callable tts_task(B, gamma) -> accuracy (negative =
+    unavailable).  Returns (B, gamma, accuracy, steps, evaluations)."""
     lib = load_library()
     cb = _TASK_FN(lambda b, g, _u: float(tts_task(b, g)))
-    B, G, acc, steps = c_int(0), c_int(0), c_double(0.0), c_int(0)
-    rc = lib.tts_greedy_search(cb, None, byref(B), byref(G), byref(acc), byref(steps))
+    B, G, acc, steps, evals = c_int(0), c_int(0), c_double(0.0), c_int(0), c_int(0)
+    rc = lib.tts_greedy_search(cb, None, _limits(max_branches, max_gamma, max_steps), byref(B), byref(G), byref(acc),
+                               byref(steps), byref(evals))
     if rc != 0:
         raise TtsError(rc, "tts_greedy_search")
-    return B.value, G.value, acc.value, steps.value
+    return B.value, G.value, acc.value, steps.value, evals.value
+
+
+def tts_grid_search(tts_task, max_branches=None, max_gamma=None):
+    """Exhaustive (B, gamma) search.  Returns (B, gamma, accuracy, evaluations)."""
+    lib = load_library()
+    cb = _TASK_FN(lambda b, g, _u: float(tts_task(b, g)))
+    B, G, acc, evals = c_int(0), c_int(0), c_double(0.0), c_int(0)
+    rc = lib.tts_grid_search(cb, None, _limits(max_branches, max_gamma, None), byref(B), byref(G), byref(acc),
+                             byref(evals))
+    if rc != 0:
+        raise TtsError(rc, "tts_grid_search")
+    return B.value, G.value, acc.value, evals.value

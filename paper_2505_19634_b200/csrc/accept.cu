@@ -101,19 +101,24 @@ __device__ __forceinline__ void draw_token(const float* __restrict__ pk, const f
         const unsigned hit = __ballot_sync(0xffffffffu, incl > t);
         int chosen = -1;
         if (hit) {
-            const int src = __ffs(hit) - 1;
+            // The first lane whose inclusive sum exceeds t holds the crossing tile, unless re-adding its
+            // tiles one by one rounds differently from the scan and leaves no crossing there: then the
+            // crossing is the first tile with mass of the next lane, so the lanes of `hit` are tried in order.
             int tile = -1;
             double base = 0.0;
-            if (lane == src) {
-                double run = incl - c;
-                for (int j = j0; j < j1; ++j) {
-                    const double nxt = run + tile_sum[j];
-                    if (nxt > t) { tile = j; base = run; break; }
-                    run = nxt;
+            for (unsigned h = hit; h != 0u && tile < 0; h &= h - 1u) {
+                const int src = __ffs(h) - 1;
+                if (lane == src) {
+                    double run = incl - c;
+                    for (int j = j0; j < j1; ++j) {
+                        const double nxt = run + tile_sum[j];
+                        if (nxt > t) { tile = j; base = run; break; }
+                        run = nxt;
+                    }
                 }
+                tile = __shfl_sync(0xffffffffu, tile, src);
+                base = __shfl_sync(0xffffffffu, base, src);
             }
-            tile = __shfl_sync(0xffffffffu, tile, src);
-            base = __shfl_sync(0xffffffffu, base, src);
             if (tile >= 0) {
                 const int x0 = tile * kTileElems + lane * 4;
                 float w[4] = {0.f, 0.f, 0.f, 0.f};

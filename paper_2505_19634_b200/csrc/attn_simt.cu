@@ -93,17 +93,10 @@ __global__ void __launch_bounds__(kThreads) attn_simt_kernel(const AttnParams p)
                 uint4 kv = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
                 if (t < n_valid) {
                     const int tok = seg.tok_begin + tok0 + t;
-                    const int page = bt[tok / kPage];
-                    bool ok = true;
-                    if (p.debug && (page < 0 || page >= p.num_pages)) {
-                        ok = false;
-                        atomicMin(p.status, (int)TTS_ERR_DEVICE_BOUNDS);
-                    }
-                    if (ok) {
-                        const size_t off = (((size_t)page * p.Hkv + seg.kvh) * kPage + tok % kPage) * kHeadDim + part * 8;
-                        kv = *reinterpret_cast<const uint4*>(p.k_pages + off);
-                        vv = *reinterpret_cast<const uint4*>(p.v_pages + off);
-                    }
+                    const int page = checked_page(p, bt, tok / kPage);
+                    const size_t off = (((size_t)page * p.Hkv + seg.kvh) * kPage + tok % kPage) * kHeadDim + part * 8;
+                    kv = *reinterpret_cast<const uint4*>(p.k_pages + off);
+                    vv = *reinterpret_cast<const uint4*>(p.v_pages + off);
                 }
                 *reinterpret_cast<uint4*>(&sm.k[t][part * 8]) = kv;
                 *reinterpret_cast<uint4*>(&sm.v[t][part * 8]) = vv;

@@ -134,13 +134,7 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 const int tok0 = t * kTile;
                 const int n_pages = ceil_div(min(kTile, seg.n_tokens - tok0), kPage);
                 int page = 0;
-                if (lane < n_pages) {
-                    page = bt[(seg.tok_begin + tok0) / kPage + lane];
-                    if (p.debug && (page < 0 || page >= p.num_pages)) {
-                        atomicMin(p.status, (int)TTS_ERR_DEVICE_BOUNDS);
-                        page = 0;
-                    }
-                }
+                if (lane < n_pages) page = checked_page(p, bt, (seg.tok_begin + tok0) / kPage + lane);
                 const int y = (page * p.Hkv + seg.kvh) * kPage;
                 // K
                 if (lane == 0) {

@@ -267,13 +267,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 const int tok0 = (cur.t + i) * kTileT;
                 const int n_pages = ceil_div(min(kTileT, seg.n_tokens - tok0), kPage);
                 int page = 0;
-                if (lane < n_pages) {
-                    page = bt[(seg.tok_begin + tok0) / kPage + lane];
-                    if (p.debug && (page < 0 || page >= p.num_pages)) {
-                        atomicMin(p.status, (int)TTS_ERR_DEVICE_BOUNDS);
-                        page = 0;
-                    }
-                }
+                if (lane < n_pages) page = checked_page(p, bt, (seg.tok_begin + tok0) / kPage + lane);
                 const int slot = ring0 + ring_pos;
                 if (lane == 0) {
                     alive = mbar_wait(bar(L::EMPTY + slot), ring_round ^ 1, ab);

@@ -1,7 +1,9 @@
 // C-ABI layer: argument checks, context and workspace management, kernel launches, and the
 // host-only helpers (answer aggregation, greedy search).  See include/tts.h for the contract.
 #include <math.h>
+#include <algorithm>
 #include <new>
+#include <vector>
 #include <stdlib.h>
 #include <string.h>
 
@@ -39,6 +41,7 @@ Plan make_plan(const Ctx* c, int nr, int n_branches) {
         pl.rb_rows = simt_rb_rows(nr); pl.tile_tokens = kSimtTileTokens; pl.grid = c->n_sms * 3;
         pl.copies = pl.copies_pre = 1;
     }
+    if (c->cfg.max_ctas > 0 && pl.grid > c->cfg.max_ctas) pl.grid = c->cfg.max_ctas;
     return pl;
 }
 
@@ -178,7 +181,7 @@ int tts_create(const tts_config* cfg, tts_ctx** out) {
     if (cfg->max_blocks_per_branch < 1 || cfg->num_pages < 1) return TTS_ERR_INVALID;
     if (cfg->out_dtype != TTS_OUT_BF16 && cfg->out_dtype != TTS_OUT_FP32) return TTS_ERR_UNSUPPORTED;
     if (cfg->attn_impl < TTS_ATTN_AUTO || cfg->attn_impl > TTS_ATTN_TCGEN05_ROW_MAJOR) return TTS_ERR_UNSUPPORTED;
-    if (!(cfg->softmax_scale >= 0.f)) return TTS_ERR_INVALID;
+    if (!(cfg->softmax_scale >= 0.f) || cfg->max_ctas < 0) return TTS_ERR_INVALID;
 
     Ctx* c = new (std::nothrow) Ctx();
     if (!c) return TTS_ERR_INVALID;
@@ -303,59 +306,109 @@ int tts_kv_rollback(tts_ctx* ctx, int32_t* branch_lens, const int32_t* accepted_
     return TTS_OK;
 }
 
-static int vote_impl(const int64_t* answers, const float* weights, int n, int mode, int64_t* winner,
-                     int* votes) {
-    if (!answers || !winner || n < 1 || (mode == 1 && !weights)) return TTS_ERR_INVALID;
-    int best = -1;
-    double best_score = 0.0;
-    if (mode == 1) {
-        for (int i = 0; i < n; ++i)
-            if (best < 0 || (double)weights[i] > best_score) { best = i; best_score = weights[i]; }
-    } else {
-        // O(n^2) on purpose: n is the number of branches (<= a few hundred), no allocation
-        for (int i = 0; i < n; ++i) {
-            bool seen = false;
-            for (int j = 0; j < i && !seen; ++j) seen = answers[j] == answers[i];
-            if (seen) continue;
-            double s = 0.0;
-            for (int j = i; j < n; ++j)
-                if (answers[j] == answers[i]) s += weights ? (double)weights[j] : 1.0;
-            if (best < 0 || s > best_score) { best = i; best_score = s; }
+// Answer aggregation.  The branches are ordered by (answer, branch index); every run of equal answers
+// is one candidate whose score is its number of branches or the sum of their weights (added in branch
+// order, fp64); the best score wins and equal scores go to the run that starts at the lowest branch.
+static int aggregate_votes(const int64_t* answers, const float* weights, int n, int64_t* winner, int* votes) {
+    if (!answers || !winner || n < 1) return TTS_ERR_INVALID;
+    std::vector<int> order(n);
+    for (int i = 0; i < n; ++i) order[i] = i;
+    std::sort(order.begin(), order.end(), [&](int a, int b) {
+        return answers[a] != answers[b] ? answers[a] < answers[b] : a < b;
+    });
+    int win_first = -1, win_count = 0;
+    double win_score = 0.0;
+    for (int lo = 0; lo < n;) {
+        int hi = lo;
+        double score = 0.0;
+        while (hi < n && answers[order[hi]] == answers[order[lo]]) {
+            score += weights ? (double)weights[order[hi]] : 1.0;
+            ++hi;
         }
+        const int first = order[lo];                      // lowest branch index of the run
+        if (win_first < 0 || score > win_score || (score == win_score && first < win_first)) {
+            win_first = first; win_score = score; win_count = hi - lo;
+        }
+        lo = hi;
     }
-    int count = 0;
-    for (int j = 0; j < n; ++j) count += answers[j] == answers[best];
-    *winner = answers[best];
-    if (votes) *votes = count;
+    *winner = answers[win_first];
+    if (votes) *votes = win_count;
     return TTS_OK;
 }
 
 int tts_majority_vote(const int64_t* answers, const float* weights, int n, int64_t* winner, int* votes) {
-    return vote_impl(answers, weights, n, 0, winner, votes);
+    return aggregate_votes(answers, weights, n, winner, votes);
 }
 
 int tts_confidence_max(const int64_t* answers, const float* weights, int n, int64_t* winner, int* votes) {
-    return vote_impl(answers, weights, n, 1, winner, votes);
+    if (!answers || !weights || !winner || n < 1) return TTS_ERR_INVALID;
+    const float* top = std::max_element(weights, weights + n);      // the first of equal maxima
+    *winner = answers[top - weights];
+    if (votes) *votes = (int)std::count(answers, answers + n, *winner);
+    return TTS_OK;
 }
 
-int tts_greedy_search(tts_task_fn tts_task, void* user, int* best_branches, int* best_gamma,
-                      double* best_acc, int* steps) {
-    if (!tts_task || !best_branches || !best_gamma) return TTS_ERR_INVALID;
-    int B = 1, gamma = 0, n_steps = 0;
-    double acc = tts_task(B, gamma, user);
-    for (;;) {
+// (B, gamma) search.  A configuration is a point of the lattice B = 1, 2, 4, .. <= max_branches,
+// gamma = 0 .. max_gamma; the caller's task function scores it (negative = not available).
+namespace {
+
+struct SearchBox { int max_branches, max_gamma, max_steps; };
+
+bool search_box(const tts_search_limits* lim, SearchBox* box) {
+    box->max_branches = lim ? lim->max_branches : 64;
+    box->max_gamma = lim ? lim->max_gamma : 7;
+    box->max_steps = lim && lim->max_steps > 0 ? lim->max_steps : 64;
+    return box->max_branches >= 1 && box->max_branches <= (1 << 20) && box->max_gamma >= 0 && box->max_gamma <= 4096;
+}
+
+struct Move { int branch_factor, gamma_step; };
+// Candidate moves in order of preference among equals: more branches first, then a longer draft.
+const Move kMoves[] = {{2, 0}, {1, 1}};
+
+}  // namespace
+
+int tts_greedy_search(tts_task_fn tts_task, void* user, const tts_search_limits* limits, int* best_branches,
+                      int* best_gamma, double* best_acc, int* steps, int* evaluations) {
+    SearchBox box;
+    if (!tts_task || !best_branches || !best_gamma || !search_box(limits, &box)) return TTS_ERR_INVALID;
+    int at_b = 1, at_g = 0, n_steps = 0, n_eval = 1;
+    double at_acc = tts_task(at_b, at_g, user);
+    while (n_steps < box.max_steps) {
         ++n_steps;
-        const double acc_b = B <= (1 << 29) ? tts_task(2 * B, gamma, user) : -1.0;
-        const double acc_g = tts_task(B, gamma + 1, user);
-        int nb, ng; double nacc;
-        if (acc_b >= acc_g) { nb = 2 * B; ng = gamma; nacc = acc_b; }
-        else                { nb = B; ng = gamma + 1; nacc = acc_g; }
-        if (nacc > acc && nacc >= 0.0) { B = nb; gamma = ng; acc = nacc; }
-        else break;
+        int to_b = 0, to_g = 0;
+        double to_acc = -1.0;
+        for (const Move& mv : kMoves) {
+            const int b = at_b * mv.branch_factor, g = at_g + mv.gamma_step;
+            if (b > box.max_branches || g > box.max_gamma) continue;      // outside the lattice: not evaluated
+            const double a = tts_task(b, g, user);
+            ++n_eval;
+            if (a >= 0.0 && a > to_acc) { to_b = b; to_g = g; to_acc = a; }
+        }
+        if (!(to_acc > at_acc)) break;                                    // no neighbour improves: local optimum
+        at_b = to_b; at_g = to_g; at_acc = to_acc;
     }
-    *best_branches = B; *best_gamma = gamma;
-    if (best_acc) *best_acc = acc;
+    *best_branches = at_b; *best_gamma = at_g;
+    if (best_acc) *best_acc = at_acc;
     if (steps) *steps = n_steps;
+    if (evaluations) *evaluations = n_eval;
+    return TTS_OK;
+}
+
+int tts_grid_search(tts_task_fn tts_task, void* user, const tts_search_limits* limits, int* best_branches,
+                    int* best_gamma, double* best_acc, int* evaluations) {
+    SearchBox box;
+    if (!tts_task || !best_branches || !best_gamma || !search_box(limits, &box)) return TTS_ERR_INVALID;
+    int win_b = 1, win_g = 0, n_eval = 0;
+    double win_acc = -1.0;
+    for (int b = 1; b <= box.max_branches; b *= 2)
+        for (int g = 0; g <= box.max_gamma; ++g) {
+            const double a = tts_task(b, g, user);
+            ++n_eval;
+            if (a >= 0.0 && a > win_acc) { win_b = b; win_g = g; win_acc = a; }   // first of equal optima in (B, gamma) order
+        }
+    *best_branches = win_b; *best_gamma = win_g;
+    if (best_acc) *best_acc = win_acc;
+    if (evaluations) *evaluations = n_eval;
     return TTS_OK;
 }
 
@@ -475,7 +528,13 @@ int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const v
     // Two more streams carry the copies that need not wait for the kernels: the queries of later layers and
     // the accept inputs go host-to-device while the first layers run, the outputs of finished layers go back
     // while later layers run.  Events order them against the context's stream, chunk of layers by chunk.
-#define TTS_CK(x) do { e = (x); if (e != cudaSuccess) return cuda_fail(c, e); } while (0)
+    // an error return must not leave copies from or to the caller's host buffers in flight
+    auto drain = [&]() {
+        cudaStreamSynchronize(c->stream);
+        if (c->h2d_stream) cudaStreamSynchronize(c->h2d_stream);
+        if (c->d2h_stream) cudaStreamSynchronize(c->d2h_stream);
+    };
+#define TTS_CK(x) do { e = (x); if (e != cudaSuccess) { drain(); return cuda_fail(c, e); } } while (0)
     if (!c->host_ev) {
         TTS_CK(cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking));
         TTS_CK(cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking));
@@ -535,7 +594,7 @@ int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const v
         for (int l = l0; l < l1; ++l) {
             int rc = tts_verify_attn(ctx, d_q + up(q_layer) * l, k_pools[l], v_pools[l], d_bt, prefix_len, d_bl,
                                      n_branches, gamma, TTS_MASK_CAUSAL, d_o + up(o_layer) * l);
-            if (rc != TTS_OK) return rc;
+            if (rc != TTS_OK) { drain(); return rc; }
         }
         TTS_CK(cudaEventRecord(ev_o[ch], st));
         TTS_CK(cudaStreamWaitEvent(down_st, ev_o[ch], 0));
@@ -544,7 +603,7 @@ int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const v
     TTS_CK(cudaStreamWaitEvent(st, ev_acc, 0));
     int rc = tts_accept(ctx, d_pt, gamma > 0 ? d_qd : nullptr, gamma > 0 ? d_dt : nullptr, d_un, n_branches, gamma,
                         vocab, d_al, d_nt);
-    if (rc != TTS_OK) return rc;
+    if (rc != TTS_OK) { drain(); return rc; }
     TTS_CK(cudaMemcpyAsync(accepted_len_host, d_al, (size_t)n_branches * 4, cudaMemcpyDeviceToHost, st));
     TTS_CK(cudaMemcpyAsync(next_token_host, d_nt, (size_t)n_branches * 4, cudaMemcpyDeviceToHost, st));
     TTS_CK(cudaStreamSynchronize(st));

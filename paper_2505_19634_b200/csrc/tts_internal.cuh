@@ -251,6 +251,19 @@ __device__ inline void piece_slot(const AttnParams& p, const SegInfo& s, int cta
     }
 }
 
+// Physical page of logical block `blk` of a block-table row.  With the debug checks on, a block
+// beyond the row or a page outside the pool raises TTS_ERR_DEVICE_BOUNDS and page 0 is read instead
+// (valid memory; the result of the call is then meaningless, the access is not out of range).
+__device__ __forceinline__ int checked_page(const AttnParams& p, const int32_t* bt_row, int blk) {
+    if (!p.debug) return bt_row[blk];
+    int page = blk >= 0 && blk < p.max_blocks ? bt_row[blk] : -1;
+    if (page < 0 || page >= p.num_pages) {
+        atomicMin(p.status, (int)TTS_ERR_DEVICE_BOUNDS);
+        page = 0;
+    }
+    return page;
+}
+
 // 64-bit visibility mask of query position i over the last R private tokens of its branch:
 // bit a set <=> row i sees token (L - R + a).  Causal: bits 0..i.  Tree: i and its ancestors.
 __device__ inline unsigned long long row_visibility(const AttnParams& p, int b, int i) {

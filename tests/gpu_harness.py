@@ -22,11 +22,11 @@ def dev(a: np.ndarray) -> torch.Tensor:
 
 
 def make_ctx(case: ti.AttnCase, impl=tts.ATTN_AUTO, out_dtype=tts.OUT_BF16, debug=False,
-             max_rows=None, max_branches=None) -> tts.TtsContext:
+             max_rows=None, max_branches=None, max_ctas=0) -> tts.TtsContext:
     s = case.shape
     return tts.TtsContext(s.n_q_heads, s.n_kv_heads, max_branches or s.n_branches,
                           max_rows or s.rows_per_branch, case.max_blocks, case.num_pages,
-                          out_dtype=out_dtype, attn_impl=impl, debug_bounds=debug)
+                          out_dtype=out_dtype, attn_impl=impl, debug_bounds=debug, max_ctas=max_ctas)
 
 
 def run_attn(case: ti.AttnCase, impl=tts.ATTN_AUTO, out_dtype=tts.OUT_BF16, tree_parents=None, debug=True,

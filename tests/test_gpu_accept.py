@@ -81,6 +81,42 @@ def test_special_cases():
         check(cc, f"zero residual u={u_last}", designed_near=True)
 
 
+def test_draw_exactly_on_a_boundary_of_the_scan(capsys):
+    """Dyadic weights (every sum exact in any order) and a uniform that puts u * Z exactly on the end of the
+    vocabulary range that one lane of the scanning warp sums, followed by tokens of zero weight: the draw is the
+    first token with weight after that boundary (running sum strictly above u * Z), in the bonus draw and in
+    the residual draw alike."""
+    V = 152064
+    per_lane = -(-(-(-V // 128)) // 32) * 128            # tokens per lane of the 32-lane scan over 128-token tiles
+    for lanes in (1, 2, 17):
+        edge = lanes * per_lane
+        w = np.zeros(V, np.float64)
+        w[5:edge:37] = 1.0                                # mass before the boundary
+        w[edge + 7::53] = 1.0                             # none in [edge, edge + 7)
+        w[w > 0] *= 2.0 ** -18
+        before = w[:edge].sum()
+        w[0] = 1.0 - w.sum()                              # total mass exactly 1, still dyadic
+        u = np.float32(w[:edge].sum())
+        assert float(u) == w[:edge].sum() and w.sum() == 1.0 and before > 0
+        p = w.astype(np.float32)
+        assert (p.astype(np.float64) == w).all()
+        # bonus draw (gamma = 0) from p
+        bonus = ti.AcceptCase(p_target=p[None, None].copy(), q_draft=np.zeros((1, 0, V), np.float32),
+                              draft_tokens=np.zeros((1, 0), np.int32), uniforms=np.array([[u]], np.float32),
+                              n_branches=1, gamma=0, vocab=V)
+        # residual draw: q takes the draft token's mass away from p, the rest of p - q is w scaled by 1/2
+        q = np.zeros(V, np.float32); q[3] = 1.0
+        pr = (w / 2).astype(np.float32); pr[3] = 0.0
+        resid = ti.AcceptCase(p_target=np.stack([pr, pr])[None].copy(), q_draft=q[None, None].copy(),
+                              draft_tokens=np.array([[3]], np.int32), uniforms=np.array([[0.5, u]], np.float32),
+                              n_branches=1, gamma=1, vocab=V)
+        for case, what in ((bonus, "bonus"), (resid, "residual")):
+            acc_o, nxt_o, _ = oracle.accept(case.p_target, case.q_draft, case.draft_tokens, case.uniforms)
+            acc_g, nxt_g = run_accept(case)
+            assert int(nxt_o[0]) == edge + 7, what       # the oracle's strict crossing
+            assert np.array_equal(acc_g, acc_o) and np.array_equal(nxt_g, nxt_o), what
+
+
 def test_lossless_chi_square_on_gpu():
     """The chi-square pin of the oracle, run through the CUDA kernel: 65536 branches per call."""
     V, per_call, calls = 16, 65536, 8

@@ -30,9 +30,10 @@ def run_tree(case, parents, check_status=True):
     return acc.cpu().numpy(), last.cpu().numpy(), nxt.cpu().numpy(), st
 
 
-@pytest.mark.parametrize("n,depth,vocab,seed", [(6, 3, 64, 1), (12, 5, 1024, 2), (30, 8, 4100, 3), (60, 10, 32768, 4), (64, 64, 132, 5)])
-def test_trees_match_oracle(n, depth, vocab, seed):
-    N = 37
+@pytest.mark.parametrize("n,depth,vocab,seed,N", [(6, 3, 64, 1, 37), (12, 5, 1024, 2, 37), (30, 8, 4100, 3, 37),
+                                                    (60, 10, 32768, 4, 37), (64, 64, 132, 5, 37),
+                                                    (60, 6, 152064, 6, 8)])        # the tree workload's own shape
+def test_trees_match_oracle(n, depth, vocab, seed, N):
     case = ti.make_accept_case(N, n, vocab, 2.0, seed=seed, draft_noise=0.6)
     parents = ti.make_tree_parents(N, n, depth, seed + 100)
     acc_o, last_o, nxt_o, near = oracle.accept_tree(case.p_target, case.q_draft, case.draft_tokens, parents, case.uniforms)

@@ -206,36 +206,91 @@ def test_debug_bounds_reports_bad_page_id_without_faulting():
     ctx.close()
 
 
-def _sampled_rows(case, n, seed):
-    s = case.shape
-    rng = np.random.default_rng(seed)
-    rows = np.stack([rng.integers(0, s.n_branches, n), rng.integers(0, s.rows_per_branch, n),
-                     rng.integers(0, s.n_q_heads, n)], axis=1).astype(np.int32)
-    # always include the first and last row of the first and last branch
-    rows[:4] = [[0, 0, 0], [0, s.gamma, s.n_q_heads - 1], [s.n_branches - 1, 0, 0],
-                [s.n_branches - 1, s.gamma, s.n_q_heads - 1]]
-    return rows
+@impl_param
+def test_debug_bounds_reports_a_block_index_past_the_table_row(impl):
+    """branch_lens lives on the device, so the host cannot see a branch that claims more tokens than its
+    block-table row holds.  With the debug checks on, the kernels notice the block index, read page 0 in
+    its place (no out-of-range access: the last branch's row ends the table) and report -4."""
+    case = ti.make_attn_case(replace(SMALL, branch_lens=(19, 3, 144)), 3)       # 144 = 9 full pages: the longest row is full
+    assert case.prefix_len + 144 == 16 * case.max_blocks
+    case.branch_lens[2] += 16                                                   # one page more than the row has
+    ctx = make_ctx(case, impl=impl, debug=True)
+    run_attn(case, ctx=ctx, check_status=False)
+    assert ctx.tts_last_status() == -4
+    assert ctx.tts_last_status() == 0
+    ctx.close()
 
 
-def _check_sampled(case, impl, rows, what):
-    want = oracle_out(case, row_sel=rows)
-    got = run_attn(case, impl, debug=False)[rows[:, 0], rows[:, 1], rows[:, 2]]
-    assert_attn_close(got, want, what=what)
+def _check_all_rows(case, impl, what, tree_parents=None, rms_gate=5e-3, out_dtype=tts.OUT_BF16, **ctx_kw):
+    """Every output row against the oracle, in the launch configuration the benchmark times (no debug checks)."""
+    kw = dict(mask_kind=1, tree_parents=tree_parents) if tree_parents is not None else {}
+    want = oracle_out(case, **kw)
+    ctx = make_ctx(case, impl, out_dtype=out_dtype, debug=False, **ctx_kw)
+    got = run_attn(case, out_dtype=out_dtype, ctx=ctx, tree_parents=tree_parents)
+    ctx.close()
+    assert_attn_close(got, want, rms_gate=rms_gate, what=what)
+    return got
 
 
-def test_32b_layer_full_size_sampled_rows():
+def test_32b_layer_full_size_all_rows():
     """One layer of the benchmark's workload at full size (16 x 4096 private + 512 prefix tokens, 258 MiB of
-    K/V), in the launch configuration bench.py times (automatic kernel choice, no debug checks), on 96
-    sampled output rows the oracle computes one by one."""
+    K/V), automatic kernel choice, no debug checks: all 2560 output rows against the oracle, so every
+    (branch, KV head) group and every piece boundary of the schedule is looked at."""
     case = ti.make_attn_case(replace(ti.CONFIGS["32b"], n_layers=1), 0x5EED + 2)
-    _check_sampled(case, tts.ATTN_AUTO, _sampled_rows(case, 96, 1), "32b layer")
+    _check_all_rows(case, tts.ATTN_AUTO, "32b layer")
 
 
-@pytest.mark.parametrize("n,gamma", [(64, 1), (7, 5)])
-def test_sweep_points_full_lengths_sampled_rows(n, gamma):
+@pytest.mark.parametrize("n,gamma", [(64, 1), (7, 5), (32, 3), (16, 5), (1, 3)])
+def test_sweep_points_full_lengths_all_rows(n, gamma):
     """Points of the branch/length sweep at full lengths (ragged 1024..8192 private tokens, prefix
-    256..1024, random page permutation), sampled rows."""
+    256..1024, random page permutation, NaN in every slot no query may read): all rows."""
     shp = ti.sweep_shape(n, gamma, seed=100 + n)
     case = ti.make_attn_case(shp, 100 + n)
     ti.poison_unused_slots(case)
-    _check_sampled(case, tts.ATTN_AUTO, _sampled_rows(case, 64, 2), shp.name)
+    _check_all_rows(case, tts.ATTN_AUTO, shp.name)
+
+
+def test_tree_config_60_node_trees_full_size():
+    """The tree-verification workload at full size: 32B layer shape, 8 branches, 60-node draft trees
+    (random parents, depth <= 6), context 8192 of which 512 shared prefix, random page permutation:
+    60 x 5 = 300 stacked rows per (branch, KV head), i.e. three 128-row blocks of the row-major kernel and
+    the general merge kernel.  All rows against the oracle's ancestor mask."""
+    shp = ti.AttnShape("tree", n_q_heads=40, n_kv_heads=8, prefix_len=512, n_branches=8, gamma=59,
+                       private_len=8192 - 512)
+    case = ti.make_attn_case(shp, 0x5EED + 5)
+    ti.poison_unused_slots(case)
+    parents = ti.make_tree_parents(8, 60, 6, seed=0x5EED + 5)
+    _check_all_rows(case, tts.ATTN_AUTO, "tree config", tree_parents=parents)
+
+
+@pytest.mark.parametrize("name,gamma,lens", [("rows_104", 12, (300, 45, 700, 13)), ("rows_160", 19, (300, 45, 700, 20)),
+                                             ("rows_512", 63, (300, 64, 700, 129))])
+def test_causal_chains_with_many_rows_per_kv_head(name, gamma, lens):
+    """Causal chains whose stacked rows per KV head exceed one 128-row block (G = 8): 104 rows (one block,
+    not replicated), 160 (two blocks), 512 (four blocks: the most a call can carry)."""
+    shp = ti.AttnShape(name, n_q_heads=16, n_kv_heads=2, prefix_len=272, n_branches=4, gamma=gamma, branch_lens=lens,
+                       extra_pages=3)
+    case = ti.make_attn_case(shp, 61)
+    ti.poison_unused_slots(case)
+    for impl in (tts.ATTN_AUTO, tts.ATTN_TCGEN05_ROW_MAJOR, tts.ATTN_SIMT):
+        _check_all_rows(case, impl, f"{name} impl {IMPL_NAMES[impl]}")
+
+
+@impl_param
+def test_split_invariance(impl):
+    """The same ragged problem with the main kernel's grid capped at 1, 7, 37 CTAs and uncapped: the KV
+    tokens are cut into different pieces each time, every result must lie inside the oracle's band and the
+    results must agree with one another to 2e-3 relative RMS (compared in fp32 output: two bf16 roundings
+    of nearly equal values differ by a whole bf16 step, 2^-9 relative, in a good part of the elements)."""
+    shp = replace(SMALL, n_q_heads=16, n_kv_heads=2, n_branches=5, gamma=3, prefix_len=400 // 16 * 16,
+                  branch_lens=(700, 4, 131, 1290, 257))
+    case = ti.make_attn_case(shp, 17)
+    ti.poison_unused_slots(case)
+    want = oracle_out(case)
+    outs = []
+    for cap in (1, 7, 37, 0):
+        _check_all_rows(case, impl, f"cap {cap}", max_ctas=cap)
+        outs.append(_check_all_rows(case, impl, f"cap {cap} fp32", out_dtype=tts.OUT_FP32, max_ctas=cap))
+    ref_rms = np.sqrt((want ** 2).mean())
+    for o in outs[1:]:
+        assert np.sqrt(((o - outs[0]) ** 2).mean()) / ref_rms <= 2e-3

@@ -67,3 +67,30 @@ def test_greedy_search_stops_at_local_optimum_and_table_edge():
     assert oracle.greedy_search(acc)[:2] == (1, 0)
     acc = np.arange(12, dtype=np.float64).reshape(3, 4)       # always improving: ends at the edge
     assert oracle.greedy_search(acc)[:2] == (4, 3)
+
+
+def test_grid_search_evaluation_count_and_optimum():
+    """56 evaluations on the paper's 7 x 8 lattice; the optimum is the table's maximum, which greedy
+    search also reaches on the unimodal surfaces of the search-comparison table (Section 4.5)."""
+    b_max, n_gamma, evals = [tuple(map(int, l.split())) for l in
+                             (GOLDEN / "grid_search_evaluations.txt").read_text().splitlines()
+                             if l and not l.startswith("#")][0]
+    n_logb = int(np.log2(b_max)) + 1
+    rows = [tuple(map(int, l.split())) for l in (GOLDEN / "greedy_search_steps.txt").read_text().splitlines()
+            if l and not l.startswith("#")]
+    for b_opt, g_opt, _ in rows:
+        lb, g = np.meshgrid(np.arange(n_logb), np.arange(n_gamma), indexing="ij")
+        acc = 90.0 - 3.0 * np.abs(lb - int(np.log2(b_opt))) - 2.0 * np.abs(g - g_opt)
+        B, gamma, best, n = oracle.grid_search(acc)
+        assert n == evals
+        assert (B, gamma) == (b_opt, g_opt) and best == acc.max()
+        assert oracle.greedy_search(acc)[:3] == (B, gamma, best)
+    # a second hill that greedy search cannot see from (1, 0): the grid finds it, greedy does not
+    acc = np.zeros((n_logb, n_gamma))
+    acc[0, 0], acc[1, 0], acc[0, 1] = 5.0, 4.0, 4.0
+    acc[5, 6] = 9.0
+    assert oracle.grid_search(acc)[:3] == (32, 6, 9.0)
+    assert oracle.greedy_search(acc)[:3] == (1, 0, 5.0)
+    # equal optima: the first in (B, gamma) order
+    acc = np.ones((3, 3))
+    assert oracle.grid_search(acc)[:2] == (1, 0)

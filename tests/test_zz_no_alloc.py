@@ -4,14 +4,15 @@ that stops at the first failure has then already run every other test).
 tts_verify_attn_noalloc is meant for hosts that cannot allocate device memory at call time, so it
 keeps its partial results in a fixed array inside the library.  That array survives between calls
 and is shared by all of them; the test therefore makes two calls in a row with DIFFERENT problems
-and checks each against tts_verify_attn on the same inputs, within the tolerance of the other
-attention tests."""
+and checks each against tts_verify_attn on the same inputs, and against the CPU oracle, within the
+tolerance of the other attention tests."""
 from dataclasses import replace
 
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2505_19634_b200 as tts
 import tts_inputs as ti
 from gpu_harness import assert_attn_close, dev, dev_bf16, run_attn
@@ -39,6 +40,8 @@ def test_two_calls_in_a_row_match_the_regular_entry_point():
         want = run_attn(case, tts.ATTN_SIMT)
         got = run_noalloc(case)
         assert_attn_close(got, want, what=case.shape.name)
+        assert_attn_close(got, oracle.verify_attn(case.q, case.k_pages, case.v_pages, case.block_table, case.prefix_len,
+                                                  case.branch_lens, case.shape.gamma), what=case.shape.name + " vs oracle")
 
 
 def test_32b_layer_fits_and_larger_problems_are_refused():
