@@ -55,8 +55,7 @@ enum { TTS_OUT_BF16 = 0, TTS_OUT_FP32 = 1 };
  * stacked query rows per KV head make it worthwhile and CUDA cores otherwise.  TCGEN05 picks
  * between the two tensor-core kernels: TOKEN_MAJOR (KV tokens on the MMA M dimension, for at most
  * 64 rows per branch and KV head: chains of gamma+1 positions) and ROW_MAJOR (query rows on M, for
- * draft trees with many nodes).  The last two force one of them; TOKEN_MAJOR takes at most 896
- * branches per call (TTS_ERR_UNSUPPORTED beyond; AUTO and TCGEN05 then use ROW_MAJOR). */
+ * draft trees with many nodes).  The last two force one of them. */
 enum { TTS_ATTN_AUTO = 0, TTS_ATTN_SIMT = 1, TTS_ATTN_TCGEN05 = 2, TTS_ATTN_TCGEN05_TOKEN_MAJOR = 3,
        TTS_ATTN_TCGEN05_ROW_MAJOR = 4 };
 
@@ -119,6 +118,24 @@ TTS_API int tts_set_stream(tts_ctx* ctx, void* cuda_stream);
 TTS_API int tts_verify_attn(tts_ctx* ctx, const void* q, const void* k_pages, const void* v_pages,
                     const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
                     int n_branches, int gamma, int mask_kind, void* out);
+
+/*
+ * The schedule of the attention calls of one verify step, built once (Section 3.1: a step is one pass
+ * through all layers over the same KV cache, so block_table and branch_lens are the same in every
+ * layer's call; the target model of Appendix A.1 has 64 layers).  tts_attn_plan works out, on the device
+ * and asynchronously on the context's stream, how the KV tokens of a call with these arguments are
+ * divided among the thread blocks, and keeps the result in the context.  Every later tts_verify_attn /
+ * tts_verify_attn_tree call with the SAME block_table and branch_lens pointers, prefix_len, n_branches
+ * and rows per branch (gamma+1, or n_nodes) then starts from those tables instead of deriving the
+ * schedule again in each launch.  The caller promises that the contents of block_table and branch_lens
+ * do not change between tts_attn_plan and those calls; after changing them (tts_kv_rollback on the same
+ * branch_lens drops the plan by itself) call tts_attn_plan again or tts_attn_plan_drop.  A call whose
+ * arguments do not match the kept plan is still correct: it builds its own schedule first (one more small
+ * launch) and drops the kept plan.  Arguments and errors as for tts_verify_attn.
+ */
+TTS_API int tts_attn_plan(tts_ctx* ctx, const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
+                  int n_branches, int rows_per_branch);
+TTS_API int tts_attn_plan_drop(tts_ctx* ctx);
 
 /*
  * Tree verification (draft token trees, as produced by tree drafters such as the EAGLE-3 draft

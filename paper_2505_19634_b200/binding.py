@@ -19,7 +19,8 @@ OUT_BF16, OUT_FP32 = 0, 1
 ATTN_AUTO, ATTN_SIMT, ATTN_TCGEN05, ATTN_TCGEN05_TOKEN_MAJOR, ATTN_TCGEN05_ROW_MAJOR = 0, 1, 2, 3, 4
 
 EXPORTED_SYMBOLS = (
-    "tts_create", "tts_destroy", "tts_set_stream", "tts_verify_attn", "tts_verify_attn_tree",
+    "tts_create", "tts_destroy", "tts_set_stream", "tts_verify_attn", "tts_verify_attn_tree", "tts_attn_plan",
+    "tts_attn_plan_drop",
     "tts_accept", "tts_majority_vote", "tts_confidence_max", "tts_greedy_search", "tts_grid_search", "tts_last_status",
     "tts_last_cuda_error", "tts_launch_count", "tts_strerror", "tts_verify_step_host",
     "tts_profile_enable", "tts_profile_read", "tts_verify_attn_noalloc", "tts_kv_append", "tts_kv_rollback", "tts_accept_tree",
@@ -70,6 +71,8 @@ def load_library() -> ctypes.CDLL:
     lib.tts_set_stream.argtypes = [vp, vp]
     lib.tts_verify_attn.argtypes = [vp, vp, vp, vp, vp, c_int, vp, c_int, c_int, c_int, vp]
     lib.tts_verify_attn_tree.argtypes = [vp, vp, vp, vp, vp, c_int, vp, vp, c_int, c_int, vp]
+    lib.tts_attn_plan.argtypes = [vp, vp, c_int, vp, c_int, c_int]
+    lib.tts_attn_plan_drop.argtypes = [vp]
     lib.tts_accept.argtypes = [vp, vp, vp, vp, vp, c_int, c_int, c_int, vp, vp]
     lib.tts_accept_tree.argtypes = [vp, vp, vp, vp, vp, vp, c_int, c_int, c_int, vp, vp, vp]
     lib.tts_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, c_int, vp, c_int, c_int]
@@ -170,6 +173,13 @@ class TtsContext:
         self._check(self._lib.tts_verify_attn(self._h, _ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(block_table),
                                               int(prefix_len), _ptr(branch_lens), int(n_branches), int(gamma),
                                               int(mask_kind), _ptr(out)), "tts_verify_attn")
+
+    def tts_attn_plan(self, block_table, prefix_len: int, branch_lens, n_branches: int, rows_per_branch: int):
+        self._check(self._lib.tts_attn_plan(self._h, _ptr(block_table), int(prefix_len), _ptr(branch_lens),
+                                            int(n_branches), int(rows_per_branch)), "tts_attn_plan")
+
+    def tts_attn_plan_drop(self):
+        self._check(self._lib.tts_attn_plan_drop(self._h), "tts_attn_plan_drop")
 
     def tts_verify_attn_tree(self, q, k_pages, v_pages, block_table, prefix_len: int, branch_lens,
                              tree_parents, n_branches: int, n_nodes: int, out):

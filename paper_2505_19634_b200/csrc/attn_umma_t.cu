@@ -9,8 +9,9 @@
 // small (NB x 256 bytes), which leaves room for a ring of 5-6 operand tiles (32 KiB each) in shared
 // memory, the depth that hides HBM latency at 4 KiB page granularity.
 //
-// One persistent CTA per SM walks its run of the global tile list (tts_internal.cuh), two tiles
-// (256 tokens) per step: the latency chain of a step (MMA -> TMEM load -> consensus -> exp -> P^T
+// One persistent CTA per SM works through its pieces (the parts of the segments of tts_internal.cuh that
+// fall into its run of the tile list), which it reads from the plan tables of attn_plan.cuh: the schedule
+// is worked out once per verify step, not in each of its 64 launches.  Two tiles (256 tokens) per step: the latency chain of a step (MMA -> TMEM load -> consensus -> exp -> P^T
 // -> MMA) is paid once for both tiles, and every thread works on two independent tokens.
 //
 //   producer warps   one for K, one for V, each with its own ring of slots (K tiles are consumed as soon
@@ -45,7 +46,7 @@
 
 #include <type_traits>
 
-#include "attn_merge.cuh"
+#include "attn_plan.cuh"
 #include "tts_internal.cuh"
 #include "umma_ptx.cuh"
 
@@ -75,8 +76,9 @@ struct Lay {
     static constexpr int kOffVis = kOffRed + 4 * NB * 4;         // u64[64]
     static constexpr int kOffLsum = kOffVis + 64 * 8;            // float[2][4][NB]: row sums of a finished piece
     static constexpr int kOffMout = kOffLsum + 2 * 4 * NB * 4;   // float[2][NB]: its row references
-    static constexpr int kOffCum = kOffMout + 2 * NB * 4;        // int[2 N + 1]: tile prefix, branch lengths
-    static constexpr int kFixedBytes = kOffCum + 1024;           // + slack for the manual 1024-B alignment
+    static constexpr int kOffPlan = kOffMout + 2 * NB * 4;       // CtaPlan: this CTA's record of the plan
+    static constexpr int kBytes = kOffPlan + (int)sizeof(CtaPlan) + 1024;   // + slack for the manual 1024-B alignment
+    static_assert(kOffPlan % 16 == 0, "the plan record is copied in 16-byte words");
     static constexpr uint32_t kTmemCols = NB == 32 ? 256 : 512;  // 2 pairs of S^T buffers + 2 O^T, power of two
     // barrier indices
     static constexpr int FULL = 0, EMPTY = kSlots, S_FULL = 2 * kSlots, S_FREE = S_FULL + 2, P_FULL = S_FREE + 2,
@@ -136,14 +138,14 @@ template <int NB, int NT>
 struct QFetch {
     static constexpr int QPT = NB * 16 / NT;
     uint4 v[QPT];
-    __device__ __forceinline__ void load(const AttnParams& p, const SegInfo& seg, int t) {
+    __device__ __forceinline__ void load(const AttnParams& p, const PieceDesc& seg, int t) {
 #pragma unroll
         for (int k = 0; k < QPT; ++k) {
             const int idx = t + k * NT, r = idx >> 4, c = idx & 15;
             v[k] = make_uint4(0, 0, 0, 0);
             if (r < seg.n_rows) {
                 int row = seg.row0 + r, b = seg.b, i, gq;
-                if (seg.kind == 0) fast_divmod(row, p.nr, b, row);
+                if (seg.kind == 0) { int db; fast_divmod(row, p.nr, db, row); b += db; }
                 fast_divmod(row, p.G, i, gq);
                 const __nv_bfloat16* src = p.q + (((size_t)b * p.R + i) * p.Hq + seg.kvh * p.G + gq) * kHeadDim;
                 v[k] = __ldg(reinterpret_cast<const uint4*>(src) + c);
@@ -163,26 +165,31 @@ struct QFetch {
 // [token half][dim half][8 tokens][128 bytes].
 __device__ __forceinline__ int tile_row_off(int row) { return (row >> 4) * 4096 + ((row >> 3) & 1) * 2048 + (row & 7) * 128; }
 
-// Walks the steps (two tiles, one at the end of a piece with an odd count) of a CTA's run of the tile list.
+// This CTA's part of the plan: its record (a copy in shared memory) and, for a CTA with more pieces than
+// the record holds, the global list.
+struct PlanView {
+    const CtaPlan* rec;
+    const PieceDesc* rest;      // plan_pieces + piece_begin
+    __device__ __forceinline__ PieceDesc piece(int i) const { return i < kPlanInline ? rec->first_pieces[i] : rest[i]; }
+    __device__ __forceinline__ int tiles(int i) const { return i < kPlanInline ? rec->first_pieces[i].n_tiles : rest[i].n_tiles; }
+};
+
+// Walks the steps (two tiles, one at the end of a piece with an odd count) of a CTA's pieces.
 struct StepCursor {
-    SegInfo seg;
-    int t, t_last;      // first tile of the step and end of the piece, as tile indices inside the segment
-    int piece;          // pieces before this one
-    int g_end;
-    bool valid, first;  // first: first step of its piece
-    __device__ void init(const SegInfo& s0, int g_begin, int g_end_) {
-        seg = s0; g_end = g_end_; piece = 0; valid = true; first = true;
-        t = g_begin - s0.tile_begin; t_last = min(s0.n_tiles, g_end_ - s0.tile_begin);
+    int piece, n_pieces;  // index of the current piece
+    int t, n_t;           // first tile of the step within the piece, tiles of the piece
+    bool valid, first;    // first: first step of its piece
+    __device__ void init(const PlanView& pv) {
+        piece = 0; n_pieces = pv.rec->n_pieces; valid = n_pieces > 0; first = true;
+        t = 0; n_t = valid ? pv.tiles(0) : 0;
     }
-    __device__ int nt() const { return min(2, t_last - t); }
-    __device__ bool last() const { return t + 2 >= t_last; }        // last step of its piece
-    __device__ void advance(const AttnParams& p, const int* cum) {
+    __device__ int nt() const { return min(2, n_t - t); }
+    __device__ bool last() const { return t + 2 >= n_t; }            // last step of its piece
+    __device__ void advance(const PlanView& pv) {
         t += 2; first = false;
-        if (t < t_last) return;
-        if (seg.tile_begin + t_last >= g_end) { valid = false; return; }
-        seg = next_segment(p, cum, seg);
-        t = 0; t_last = min(seg.n_tiles, g_end - seg.tile_begin);
-        ++piece; first = true;
+        if (t < n_t) return;
+        if (++piece >= n_pieces) { valid = false; return; }
+        n_t = pv.tiles(piece); t = 0; first = true;
     }
 };
 
@@ -202,11 +209,13 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     const uint32_t bar0 = sbase + L::kOffBar;
     auto bar = [&](int i) { return bar0 + 8u * i; };
     volatile int* misc = reinterpret_cast<volatile int*>(smem + L::kOffMisc);   // [0] abort flag, [1] tmem base
-    int* cum = reinterpret_cast<int*>(smem + L::kOffCum);
+    const CtaPlan* rec = reinterpret_cast<const CtaPlan*>(smem + L::kOffPlan);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Abort ab{misc, p.status};
 
-    // ---- set-up that needs no input first: barriers, TMEM, tensor-map prefetch; then the run of this CTA ----
+    // ---- set-up: barriers, TMEM, tensor-map prefetch, and this CTA's record of the plan (one coalesced read) ----
+    if (tid >= 32 && tid < 64)
+        reinterpret_cast<uint4*>(smem + L::kOffPlan)[tid - 32] = __ldg(reinterpret_cast<const uint4*>(p.plan_cta + blockIdx.x) + (tid - 32));
     if (tid == 0) {
         misc[0] = 0;
         for (int i = 0; i < NS; ++i) { mbar_init(bar(L::FULL + i), 1); mbar_init(bar(L::EMPTY + i), 1); }
@@ -227,26 +236,14 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     if (warp == kProducerWarp + 1 && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
     fence_proxy_async();
     tc_fence_before();
-    build_branch_tile_prefix(p, cum);                      // synchronises the CTA
+    __syncthreads();
     tc_fence_after();
     const uint32_t tmem = (uint32_t)misc[1];
-    const int total = total_tiles(p, cum);
-    const int tpc = ceil_div(total, p.grid);
-    const int g_begin = blockIdx.x * tpc;
-    const int g_end = min(total, g_begin + tpc);
-    const bool has_work = g_begin < g_end;                 // uniform
+    const PlanView pv{rec, p.plan_pieces + rec->piece_begin};
+    const int n_pieces = rec->n_pieces;
+    const bool has_work = n_pieces > 0;                    // uniform
     // S^T of tile i of step ss at columns [(2 (ss & 1) + i) NB, +NB); O^T of piece pc at [(4 + (pc & 1)) NB, +NB)
     const uint32_t tmem_o0 = tmem + 4u * NB;
-    const int group0 = group_of_tile_block(p, cum, has_work ? g_begin : 0);         // synchronises the CTA
-    SegInfo seg0;
-    if (has_work) seg0 = segment_in_group(p, cum, group0, g_begin);
-
-    // Where the partial results of every group (branch, KV head) lie, for the merge kernel: a function of the
-    // schedule alone; the first epilogue warp, idle until the first piece ends, writes it for the groups that
-    // fall to this CTA (five lanes per group, one per entry).
-    if (warp == kEpilogueWarp && p.group_desc && lane < kMaxPrivBlocks + kMaxPreBlocks)
-        for (int grp = blockIdx.x; grp < p.N * p.Hkv; grp += gridDim.x)
-            group_describe_entry(p, cum, tpc, grp / p.Hkv, grp % p.Hkv, lane, static_cast<GroupDesc*>(p.group_desc)[grp]);
     if (!has_work) {
         // nothing to do for this CTA
     } else if (warp == kProducerWarp || warp == kProducerWarp + 1) {
@@ -258,16 +255,16 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         int ring_pos = 0, ring_round = 0;                   // u % ring_n, (u / ring_n) & 1, kept without dividing
         bool alive = true;
         const uint64_t stream_once = l2_policy_evict_first();
-        StepCursor cur;
-        for (cur.init(seg0, g_begin, g_end); cur.valid && alive; cur.advance(p, cum)) {
-            const SegInfo& seg = cur.seg;
-            const int32_t* bt = p.block_table + (size_t)(seg.kind == 0 ? 0 : seg.b) * p.max_blocks;
-            const int nt = cur.nt();
-            for (int i = 0; i < nt && alive; ++i, ++u) {
-                const int tok0 = (cur.t + i) * kTileT;
-                const int n_pages = ceil_div(min(kTileT, seg.n_tokens - tok0), kPage);
-                int page = 0;
-                if (lane < n_pages) page = checked_page(p, bt, (seg.tok_begin + tok0) / kPage + lane);
+        for (int pi = 0; pi < n_pieces && alive; ++pi) {
+            const PieceDesc pc = pv.piece(pi);
+            const int32_t* bt = p.block_table + (size_t)pc.bt_row * p.max_blocks;
+            for (int i = 0; i < pc.n_tiles && alive; ++i, ++u) {
+                const int tok0 = (pc.tile0 + i) * kTileT;
+                const int n_pages = ceil_div(min(kTileT, pc.seg_tokens - tok0), kPage);
+                int page_head = 0;                             // page * Hkv + kvh: the TMA coordinate of a page-head tile
+                if (lane < n_pages)
+                    page_head = u < 2 ? rec->first_pages[u * 8 + lane]
+                                      : checked_page(p, bt, (pc.tok_begin + tok0) / kPage + lane) * p.Hkv + pc.kvh;
                 const int slot = ring0 + ring_pos;
                 if (lane == 0) {
                     alive = mbar_wait(bar(L::EMPTY + slot), ring_round ^ 1, ab);
@@ -275,7 +272,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 }
                 alive = __shfl_sync(0xffffffffu, alive, 0);
                 if (alive && lane < n_pages)
-                    tma_load_page(sbase + L::kOffRing + slot * kSlotBytes + lane * 4096, tm, page * p.Hkv + seg.kvh,
+                    tma_load_page(sbase + L::kOffRing + slot * kSlotBytes + lane * 4096, tm, page_head,
                                   bar(L::FULL + slot), stream_once);
                 if (++ring_pos == ring_n) { ring_pos = 0; ring_round ^= 1; }
             }
@@ -346,17 +343,17 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
             };
             // the scores run one step ahead of the accumulation, across piece boundaries too
             StepCursor cq, cp;
-            cq.init(seg0, g_begin, g_end); cp = cq;
+            cq.init(pv); cp = cq;
             alive = issue_qk(cq);
-            cq.advance(p, cum);
+            cq.advance(pv);
             while (alive && cp.valid) {
                 if (cq.valid) {
                     alive = issue_qk(cq);
                     if (!alive) break;
-                    cq.advance(p, cum);
+                    cq.advance(pv);
                 }
                 alive = issue_pv(cp);
-                cp.advance(p, cum);
+                cp.advance(pv);
             }
         }
     } else if (warp >= kEpilogueWarp) {
@@ -366,13 +363,18 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         const float* lsum = reinterpret_cast<const float*>(smem + L::kOffLsum);
         const float* mout = reinterpret_cast<const float*>(smem + L::kOffMout);
-        SegInfo seg = seg0;
         bool alive = true;
-        for (int pc = 0, g = g_begin; alive; ++pc) {
-            const int t_last = min(seg.n_tiles, g_end - seg.tile_begin);
+        for (int pc = 0; pc < n_pieces && alive; ++pc) {
+            const PieceDesc seg = pv.piece(pc);
             const int pb = pc & 1, n_rows = seg.n_rows;
             float* po; float2* pml;
-            piece_slot(p, seg, blockIdx.x, po, pml);
+            if (seg.kind == 0) {
+                po = p.part_o_pre + (size_t)seg.slot * p.pre_stride * kHeadDim;
+                pml = p.part_ml_pre + (size_t)seg.slot * p.pre_stride;
+            } else {
+                po = p.part_o_priv + (size_t)seg.slot * p.priv_stride * kHeadDim;
+                pml = p.part_ml_priv + (size_t)seg.slot * p.priv_stride;
+            }
             alive = mbar_wait(bar(L::L_FULL + pb), (pc >> 1) & 1, ab) && mbar_wait(bar(L::O_FULL + pb), (pc >> 1) & 1, ab);
             alive = __all_sync(0xffffffffu, alive);
             if (!alive) break;
@@ -392,9 +394,6 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
             tc_fence_before();
             warp_arrive(bar(L::O_FREE + pb), lane);
             warp_arrive(bar(L::L_FREE + pb), lane);
-            g = seg.tile_begin + t_last;
-            if (g >= g_end) break;
-            seg = next_segment(p, cum, seg);
         }
     } else {
         // =========================== softmax warps ===========================
@@ -426,7 +425,7 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         float* mout = reinterpret_cast<float*>(smem + L::kOffMout);
         int ss = 0, u_v = 0, pc = 0;                          // steps, V tiles and pieces of this CTA so far
         bool ok = true;
-        SegInfo seg = seg0;
+        PieceDesc seg = pv.piece(0);
         QFetch<NB, NT> qf;
         qf.load(p, seg, tid);
         qf.store(smem + L::kOffQ, tid);
@@ -434,18 +433,16 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         warp_arrive(bar(L::Q_FULL), lane);
 
         for (;;) {
-            const int t_first = g_begin > seg.tile_begin ? g_begin - seg.tile_begin : 0;
-            const int t_last = min(seg.n_tiles, g_end - seg.tile_begin);
-            const int n_steps = ceil_div(t_last - t_first, 2);
-            const int Ltok = seg.n_tokens;
+            const int t_first = seg.tile0, t_last = seg.tile0 + seg.n_tiles;
+            const int n_steps = ceil_div(seg.n_tiles, 2);
+            const int Ltok = seg.seg_tokens;
             const int tail0 = seg.kind == 1 ? Ltok - p.R : Ltok;     // first token that needs the row mask
             const int n_rows = seg.n_rows;                            // chunks starting at or past it are skipped
             const uint32_t tmem_o = tmem_o0 + (uint32_t)((pc & 1) * NB);
-            const int g_next = seg.tile_begin + t_last;
-            const bool have_next = g_next < g_end;
-            SegInfo next = seg;
+            const bool have_next = pc + 1 < n_pieces;
+            PieceDesc next = seg;
             if (have_next) {
-                next = next_segment(p, cum, seg);
+                next = pv.piece(pc + 1);
                 qf.load(p, next, tid);                                // in flight while this piece is computed
             }
             float l_part[NCK][4];
@@ -708,15 +705,13 @@ done:
 
 template <int NB, int CG>
 cudaError_t launch_nb(Ctx* c, const AttnParams& p, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t st) {
-    const int smem = Lay<NB>::kFixedBytes + (2 * p.N + 1) * (int)sizeof(int);
     static bool attr_set[64] = {};                          // the attribute is per device
     if (c->device < 0 || c->device >= 64 || !attr_set[c->device]) {
-        cudaError_t err = cudaFuncSetAttribute(attn_umma_t_kernel<NB, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               Lay<NB>::kFixedBytes + (2 * kUmmaTMaxBranches + 1) * (int)sizeof(int));
+        cudaError_t err = cudaFuncSetAttribute(attn_umma_t_kernel<NB, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<NB>::kBytes);
         if (err != cudaSuccess) return err;
         if (c->device >= 0 && c->device < 64) attr_set[c->device] = true;
     }
-    attn_umma_t_kernel<NB, CG><<<p.grid, 128 * CG + 224, smem, st>>>(p, mk, mv);
+    attn_umma_t_kernel<NB, CG><<<p.grid, 128 * CG + 224, Lay<NB>::kBytes, st>>>(p, mk, mv);
     return cudaGetLastError();
 }
 

@@ -7,6 +7,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include "attn_plan.cuh"
 #include "tts_internal.cuh"
 
 using namespace tts;
@@ -29,7 +30,7 @@ Plan make_plan(const Ctx* c, int nr, int n_branches) {
     if (impl == TTS_ATTN_AUTO) impl = umma_available() && nr >= kUmmaMinRows ? TTS_ATTN_TCGEN05 : TTS_ATTN_SIMT;
     // few rows per KV head: KV tokens on the MMA M dimension; many (draft trees): query rows on M
     if (impl == TTS_ATTN_TCGEN05)
-        impl = nr <= kUmmaTMaxRows && n_branches <= kUmmaTMaxBranches ? TTS_ATTN_TCGEN05_TOKEN_MAJOR : TTS_ATTN_TCGEN05_ROW_MAJOR;
+        impl = nr <= kUmmaTMaxRows ? TTS_ATTN_TCGEN05_TOKEN_MAJOR : TTS_ATTN_TCGEN05_ROW_MAJOR;
     pl.impl = impl;
     if (impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR) {
         pl.rb_rows = umma_t_rows(nr); pl.tile_tokens = kUmmaTileTokens; pl.grid = c->n_sms;
@@ -48,6 +49,7 @@ Plan make_plan(const Ctx* c, int nr, int n_branches) {
 void free_workspace(Ctx* c) {
     cudaFree(c->part_o_pre); cudaFree(c->part_ml_pre); cudaFree(c->part_o_priv); cudaFree(c->part_ml_priv);
     cudaFree(c->group_desc); c->group_desc = nullptr;
+    cudaFree(c->plan_cta); cudaFree(c->plan_pieces); c->plan_cta = nullptr; c->plan_pieces = nullptr;
     c->part_o_pre = c->part_o_priv = nullptr; c->part_ml_pre = c->part_ml_priv = nullptr;
     c->pre_rows = c->priv_rows = 0;
 }
@@ -86,48 +88,45 @@ cudaError_t alloc_workspace(Ctx* c) {
     if ((e = cudaMalloc(&c->part_o_priv, priv * kHeadDim * sizeof(float))) != cudaSuccess) return e;
     if ((e = cudaMalloc(&c->part_ml_priv, priv * sizeof(float2))) != cudaSuccess) return e;
     c->pre_rows = pre; c->priv_rows = priv;
-    return cudaMalloc(&c->group_desc, (size_t)f.max_branches * f.n_kv_heads * 64);   // a GroupDesc is 48 bytes
+    if ((e = cudaMalloc(&c->group_desc, (size_t)f.max_branches * f.n_kv_heads * 64)) != cudaSuccess) return e;   // a GroupDesc is 48 bytes
+    // plan of the token-major kernel (row blocks of 32 rows): one piece per segment and one more per CTA
+    const size_t rb = (size_t)umma_t_rows(nr);
+    const size_t n_seg = (size_t)f.max_branches * f.n_kv_heads * ((nr + rb - 1) / rb) +
+                         (size_t)f.n_kv_heads * (((size_t)f.max_branches * nr + rb - 1) / rb);
+    c->plan_pieces_cap = n_seg + (size_t)c->n_sms;
+    if ((e = cudaMalloc(&c->plan_cta, (size_t)c->n_sms * sizeof(CtaPlan))) != cudaSuccess) return e;
+    return cudaMalloc(&c->plan_pieces, c->plan_pieces_cap * sizeof(PieceDesc));
 }
 
-int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
-                const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
-                const int32_t* tree_parents, int n_branches, int rows, void* out) {
-    if (!c || !q || !k_pages || !v_pages || !block_table || !branch_lens || !out) return TTS_ERR_INVALID;
+// Checks the arguments that describe the schedule of an attention call and fills the parameters that
+// depend on them (everything but q, K/V and out).
+int attn_setup(Ctx* c, const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
+               const int32_t* tree_parents, int n_branches, int rows, AttnParams* out_p, Plan* out_pl) {
+    if (!c || !block_table || !branch_lens) return TTS_ERR_INVALID;
     const tts_config& f = c->cfg;
     if (n_branches < 1 || n_branches > f.max_branches) return TTS_ERR_INVALID;
     if (rows < 1 || rows > f.max_rows_per_branch) return TTS_ERR_INVALID;
-    if (tree_parents && rows > kMaxTreeRows) return TTS_ERR_UNSUPPORTED;
-    if (!tree_parents && rows > kMaxTreeRows) return TTS_ERR_UNSUPPORTED;
+    if (rows > kMaxTreeRows) return TTS_ERR_UNSUPPORTED;
     if (prefix_len < 0 || prefix_len % f.page_size != 0) return TTS_ERR_INVALID;
     if (prefix_len / f.page_size > f.max_blocks_per_branch) return TTS_ERR_INVALID;
-    if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(out) ||
-        (reinterpret_cast<uintptr_t>(block_table) & 3u) || (reinterpret_cast<uintptr_t>(branch_lens) & 3u))
-        return TTS_ERR_INVALID;
+    if ((reinterpret_cast<uintptr_t>(block_table) & 3u) || (reinterpret_cast<uintptr_t>(branch_lens) & 3u)) return TTS_ERR_INVALID;
 
     const int G = f.n_q_heads / f.n_kv_heads;
     const int nr = rows * G;
     const Plan pl = make_plan(c, nr, n_branches);
-    if (pl.impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR && n_branches > kUmmaTMaxBranches) return TTS_ERR_UNSUPPORTED;   // only when asked for by name
-
     {
         size_t need_pre, need_priv;
         workspace_rows(n_branches, f.n_kv_heads, nr, pl.rb_rows, pl.copies, pl.copies_pre, pl.grid, &need_pre, &need_priv);
         if (need_pre > c->pre_rows || need_priv > c->priv_rows) return TTS_ERR_INVALID;
     }
-    cudaError_t e;
-
-    AttnParams p;
+    AttnParams& p = *out_p;
     memset(&p, 0, sizeof p);
-    p.q = static_cast<const __nv_bfloat16*>(q);
-    p.k_pages = static_cast<const __nv_bfloat16*>(k_pages);
-    p.v_pages = static_cast<const __nv_bfloat16*>(v_pages);
     p.block_table = block_table; p.branch_lens = branch_lens; p.tree_parents = tree_parents;
-    p.out = out;
     p.part_o_pre = c->part_o_pre; p.part_ml_pre = c->part_ml_pre;
     p.part_o_priv = c->part_o_priv; p.part_ml_priv = c->part_ml_priv;
     p.status = c->d_status;
-    // the token-major kernel tells the merge kernel where every group's partial results lie
-    p.group_desc = pl.impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR ? c->group_desc : nullptr;
+    // the token-major kernel and its merge kernel run from the plan tables
+    if (pl.impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR) { p.group_desc = c->group_desc; p.plan_cta = c->plan_cta; p.plan_pieces = c->plan_pieces; }
     p.N = n_branches; p.R = rows; p.Hq = f.n_q_heads; p.Hkv = f.n_kv_heads; p.G = G; p.nr = nr;
     p.P = prefix_len; p.max_blocks = f.max_blocks_per_branch; p.num_pages = f.num_pages;
     p.rb_rows = pl.rb_rows;
@@ -141,11 +140,41 @@ int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
     p.tile_tokens = pl.tile_tokens;
     p.tiles_pre = ceil_div(prefix_len, pl.tile_tokens);
     p.grid = pl.grid;
-    p.lens_smem = pl.impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR ? 1 : 0;
     p.out_dtype = f.out_dtype; p.debug = f.debug_bounds;
     const float scale = f.softmax_scale > 0.f ? f.softmax_scale : 1.0f / sqrtf((float)f.head_dim);
     p.scale_log2 = scale * 1.4426950408889634f;
+    *out_pl = pl;
+    return TTS_OK;
+}
 
+// Does the plan in the context's tables, built by tts_attn_plan, describe this call?
+bool plan_matches(const Ctx* c, const int32_t* block_table, int prefix_len, const int32_t* branch_lens, int n_branches, int rows) {
+    return c->plan_explicit && c->plan_key.block_table == block_table && c->plan_key.branch_lens == branch_lens &&
+           c->plan_key.prefix_len == prefix_len && c->plan_key.n_branches == n_branches && c->plan_key.rows == rows;
+}
+
+int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
+                const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
+                const int32_t* tree_parents, int n_branches, int rows, void* out) {
+    if (!c || !q || !k_pages || !v_pages || !out) return TTS_ERR_INVALID;
+    if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(out)) return TTS_ERR_INVALID;
+    AttnParams p;
+    Plan pl;
+    const int rc = attn_setup(c, block_table, prefix_len, branch_lens, tree_parents, n_branches, rows, &p, &pl);
+    if (rc != TTS_OK) return rc;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k_pages = static_cast<const __nv_bfloat16*>(k_pages);
+    p.v_pages = static_cast<const __nv_bfloat16*>(v_pages);
+    p.out = out;
+    cudaError_t e;
+
+    if (pl.impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR && !plan_matches(c, block_table, prefix_len, branch_lens, n_branches, rows)) {
+        // no plan from tts_attn_plan for these arguments: build one for this call alone
+        c->plan_explicit = 0;
+        e = launch_attn_plan(p, c->stream);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        c->launches += 1;
+    }
     const bool prof = c->profiling && c->prof_ev && c->prof_n < kProfMaxCalls;
     cudaEvent_t* ev = prof ? c->prof_ev + 3 * c->prof_n : nullptr;
     if (prof) cudaEventRecord(ev[0], c->stream);
@@ -248,6 +277,31 @@ int tts_verify_attn_tree(tts_ctx* ctx, const void* q, const void* k_pages, const
                        branch_lens, tree_parents, n_branches, n_nodes, out);
 }
 
+int tts_attn_plan(tts_ctx* ctx, const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
+                  int n_branches, int rows_per_branch) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    AttnParams p;
+    Plan pl;
+    const int rc = attn_setup(c, block_table, prefix_len, branch_lens, nullptr, n_branches, rows_per_branch, &p, &pl);
+    if (rc != TTS_OK) return rc;
+    c->plan_explicit = 0;
+    if (pl.impl != TTS_ATTN_TCGEN05_TOKEN_MAJOR) return TTS_OK;      // the other kernels derive their schedule themselves
+    const cudaError_t e = launch_attn_plan(p, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->launches += 1;
+    c->plan_key.block_table = block_table; c->plan_key.branch_lens = branch_lens;
+    c->plan_key.prefix_len = prefix_len; c->plan_key.n_branches = n_branches; c->plan_key.rows = rows_per_branch;
+    c->plan_explicit = 1;
+    return TTS_OK;
+}
+
+int tts_attn_plan_drop(tts_ctx* ctx) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c) return TTS_ERR_INVALID;
+    c->plan_explicit = 0;
+    return TTS_OK;
+}
+
 int tts_accept(tts_ctx* ctx, const float* p_target, const float* q_draft, const int32_t* draft_tokens,
                const float* uniforms, int n_branches, int gamma, int vocab, int32_t* accepted_len,
                int32_t* next_token) {
@@ -300,6 +354,7 @@ int tts_kv_rollback(tts_ctx* ctx, int32_t* branch_lens, const int32_t* accepted_
     Ctx* c = reinterpret_cast<Ctx*>(ctx);
     if (!c || !branch_lens || !accepted_len) return TTS_ERR_INVALID;
     if (n_branches < 1 || n_branches > c->cfg.max_branches || gamma < 0) return TTS_ERR_INVALID;
+    if (c->plan_explicit && c->plan_key.branch_lens == branch_lens) c->plan_explicit = 0;   // the lengths change
     cudaError_t e = launch_kv_rollback(branch_lens, accepted_len, n_branches, gamma, c->d_status, c->stream);
     if (e != cudaSuccess) return cuda_fail(c, e);
     c->launches += 1;
@@ -587,6 +642,11 @@ int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const v
     }
     TTS_CK(cudaMemcpyAsync(d_un, uniforms_host, (size_t)n_branches * (gamma + 1) * 4, cudaMemcpyHostToDevice, up_st));
     TTS_CK(cudaEventRecord(ev_acc, up_st));
+    // one schedule serves all layers
+    {
+        const int rc = tts_attn_plan(ctx, d_bt, prefix_len, d_bl, n_branches, gamma + 1);
+        if (rc != TTS_OK) { drain(); return rc; }
+    }
     // the layers, chunk by chunk; every finished chunk's outputs go back beside the next chunk's kernels
     for (int ch = 0; ch < n_chunks; ++ch) {
         const int l0 = ch * per_chunk, l1 = l0 + per_chunk < n_layers ? l0 + per_chunk : n_layers;
@@ -606,6 +666,7 @@ int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const v
     if (rc != TTS_OK) { drain(); return rc; }
     TTS_CK(cudaMemcpyAsync(accepted_len_host, d_al, (size_t)n_branches * 4, cudaMemcpyDeviceToHost, st));
     TTS_CK(cudaMemcpyAsync(next_token_host, d_nt, (size_t)n_branches * 4, cudaMemcpyDeviceToHost, st));
+    c->plan_explicit = 0;                                   // the staging buffers' contents change with the next call
     TTS_CK(cudaStreamSynchronize(st));
     TTS_CK(cudaStreamSynchronize(down_st));
     TTS_CK(cudaStreamSynchronize(up_st));

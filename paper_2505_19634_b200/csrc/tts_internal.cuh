@@ -30,6 +30,8 @@ constexpr int kMaxBranches = 1024;
 // segments of either kind and CTAs both advance along the list, (segment index within its kind +
 // CTA) is a unique index for every piece, so no scan over pieces is needed to place them in the
 // workspace.
+struct CtaPlan;
+struct PieceDesc;
 struct AttnParams {
     const __nv_bfloat16* q;
     const __nv_bfloat16* k_pages;
@@ -43,7 +45,9 @@ struct AttnParams {
     float* part_o_priv;   // [N*Hkv*n_rb_priv + grid][priv_stride][128]
     float2* part_ml_priv;
     int32_t* status;      // device status word
-    void* group_desc;     // [N*Hkv] GroupDesc (attn_merge.cuh) written by the main kernel for the merge kernel, or null
+    void* group_desc;     // [N*Hkv] GroupDesc (attn_merge.cuh) for the merge kernel: part of the plan, or null
+    const CtaPlan* plan_cta;        // [grid] the plan the token-major kernel runs from (attn_plan.cuh)
+    const PieceDesc* plan_pieces;
     int N, R, Hq, Hkv, G, nr;      // nr = R*G rows per (branch, kv head)
     int P;                          // prefix tokens
     int max_blocks, num_pages;
@@ -290,6 +294,11 @@ struct Ctx {
     float* part_o_pre; float2* part_ml_pre; float* part_o_priv; float2* part_ml_priv;
     size_t pre_rows, priv_rows;       // allocated partial rows (each 128 fp32 + one float2)
     void* group_desc;                 // one merge descriptor per (branch, KV head)
+    // plan of the token-major kernel (attn_plan.cuh): one record per CTA, the list of all pieces
+    CtaPlan* plan_cta; PieceDesc* plan_pieces; size_t plan_pieces_cap;
+    // the arguments the plan in the tables was built from by tts_attn_plan (valid while plan_explicit is set)
+    struct { const int32_t* block_table; const int32_t* branch_lens; int prefix_len, n_branches, rows; } plan_key;
+    int plan_explicit;
     // staging for the host entry point
     void* stage; size_t stage_bytes;
     cudaStream_t h2d_stream, d2h_stream;   // copies of the host entry point that overlap the kernels (created on first use)
@@ -331,7 +340,6 @@ int umma_copies(int nr);              // replication factor of a private piece's
 cudaError_t launch_attn_umma(Ctx* c, const AttnParams& p, cudaStream_t st);
 // token-major tcgen05 kernel (KV tokens on the MMA M dimension): row blocks of 32 or 64 stacked rows
 constexpr int kUmmaTMaxRows = 64;
-constexpr int kUmmaTMaxBranches = 896;   // its shared memory holds 2N + 1 schedule words beside the operand ring
 constexpr int kUmmaTGroups = 1;        // partial results a piece leaves per row
 int umma_t_rows(int nr);
 cudaError_t launch_attn_umma_t(Ctx* c, const AttnParams& p, cudaStream_t st);

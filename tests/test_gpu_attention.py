@@ -71,18 +71,61 @@ def test_edge_shapes(impl, name):
     assert_attn_close(run_attn(case, impl), oracle_out(case), what=name)
 
 
-def test_more_branches_than_the_token_major_kernel_takes():
-    """Above 896 branches the token-major kernel's shared memory cannot hold the schedule: AUTO and
-    TCGEN05 go to the row-major kernel, asking for TOKEN_MAJOR by name is refused."""
+@impl_param
+def test_900_short_branches(impl):
+    """Many short branches: every (branch, KV head) segment is a single tile, so a thread block of the
+    token-major kernel works through more pieces than its plan record holds inline."""
     n = 900
     shp = replace(SMALL, n_branches=n, gamma=2, prefix_len=16, branch_lens=tuple(3 + (7 * i) % 23 for i in range(n)))
     case = ti.make_attn_case(shp, 11)
-    want = oracle_out(case)
-    for impl in (tts.ATTN_AUTO, tts.ATTN_TCGEN05):
-        assert_attn_close(run_attn(case, impl), want, what=f"900 branches impl {impl}")
-    with pytest.raises(tts.TtsError) as e:
-        run_attn(case, tts.ATTN_TCGEN05_TOKEN_MAJOR)
-    assert e.value.status == -2                        # TTS_ERR_UNSUPPORTED
+    assert_attn_close(run_attn(case, impl), oracle_out(case), what="900 branches")
+
+
+def test_explicit_plan_is_reused_and_dropped():
+    """tts_attn_plan once, then several layers (different K/V/Q, same table and lengths): same results as
+    calls that plan for themselves, one launch fewer per call; a call with other arguments still works."""
+    import torch
+    from gpu_harness import dev, dev_bf16
+    shp = replace(SMALL, n_q_heads=16, n_kv_heads=2, n_branches=6, gamma=3, branch_lens=(700, 4, 131, 1290, 257, 64))
+    layers = [ti.make_attn_case(shp, 23, layer=l) for l in range(3)]
+    ctx = make_ctx(layers[0], tts.ATTN_TCGEN05_TOKEN_MAJOR, debug=True)
+    bt, bl = dev(layers[0].block_table), dev(layers[0].branch_lens)
+    dev_in = [(dev_bf16(c.q), dev_bf16(c.k_pages), dev_bf16(c.v_pages)) for c in layers]
+
+    def run_layers():
+        nonlocal bl
+        outs = []
+        for q, k, v in dev_in:
+            out = torch.full(q.shape, float("nan"), device="cuda", dtype=torch.bfloat16)
+            ctx.tts_verify_attn(q, k, v, bt, shp.prefix_len, bl, shp.n_branches, shp.gamma, tts.MASK_CAUSAL, out)
+            outs.append(out)
+        torch.cuda.synchronize()
+        return [o.float().cpu().numpy().astype(np.float64) for o in outs]
+
+    n0 = ctx.tts_launch_count()
+    unplanned = run_layers()
+    n1 = ctx.tts_launch_count()
+    ctx.tts_attn_plan(bt, shp.prefix_len, bl, shp.n_branches, shp.gamma + 1)
+    n2 = ctx.tts_launch_count()
+    planned = run_layers()
+    n3 = ctx.tts_launch_count()
+    assert n1 - n0 == 3 * 3 and n2 - n1 == 1 and n3 - n2 == 3 * 2
+    for c, a, b in zip(layers, unplanned, planned):
+        assert np.array_equal(a, b)
+        assert_attn_close(b, oracle_out(c), what="planned layer")
+    # other arguments (a copy of the lengths at another address): the kept plan does not apply, every call
+    # plans for itself again and the kept plan is dropped
+    bl_kept, bl = bl, bl.clone()
+    n4 = ctx.tts_launch_count()
+    again = run_layers()
+    assert ctx.tts_launch_count() - n4 == 3 * 3
+    bl = bl_kept
+    run_layers()
+    assert ctx.tts_launch_count() - n4 == 2 * 3 * 3
+    for a, b in zip(again, planned):
+        assert np.array_equal(a, b)
+    assert ctx.tts_last_status() == 0
+    ctx.close()
 
 
 @impl_param
