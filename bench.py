@@ -3,26 +3,35 @@
 accept/resample pass) on the Qwen2.5-32B-shaped workload: N=16 branches, gamma=3, prefix 512,
 4096 private tokens per branch, vocab 152064.  Prints ONE JSON line.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 32b|3b|tiny]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--config 32b|3b|tiny|tree|sweep]
 
 * value   = unique KV bytes + accept probability bytes of one step / device time of the step (GB/s),
-            inputs resident in HBM; us_per_layer is reported beside it.
+            inputs resident in HBM; us_per_layer is reported beside it.  A step is: one schedule
+            (tts_attn_plan), one attention call per layer, one accept pass; the timed steps replay one
+            CUDA graph of exactly those calls.
 * e2e     = same bytes / time of tts_verify_step_host (pinned host q/out/probabilities copied inside
             the timed region; the KV cache is device-resident state).
-* roofline= the attention main kernel: unique KV bytes of one layer / its CUDA-event duration,
-            against the measured copy bandwidth of MEASURED_PEAKS.json.
+* roofline= the attention main kernel: unique KV bytes of one layer / the time per layer of a graph of
+            the attention calls alone (an upper bound for the kernel's duration, in the launch mode of the
+            timed steps), against the measured copy bandwidth of MEASURED_PEAKS.json; for --config tree
+            the flops against the measured bf16 GEMM rate.
 * cpu_baseline = the CPU oracle timed on a bounded sample (whole layers + the accept pass).
+--config sweep runs the branch / draft-length sweep (N x gamma x 3 seeds, ragged lengths), checks every
+point against the oracle and prints a table before the JSON line.
 With --gpus N > 1 (under torchrun) every rank runs an independent replica of the step (the path
 has no exchange step); value sums the ranks' bytes over the slowest rank's time.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
 import sys
 import time
+from dataclasses import replace
 from pathlib import Path
 
 import numpy as np
@@ -34,14 +43,42 @@ import tts_inputs as ti  # noqa: E402
 
 METRIC = "verify-step µs/layer and KV HBM GB/s vs peak at N branches × (γ+1) tokens"
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1400.0          # sustained
+NOMINAL_HBM_GBS = 8000.0               # the nominal HBM3e figure the 70 % target is also quoted against
+L2_BYTES = 132_000_000
+
+TREE = ti.AttnShape("tree", n_q_heads=40, n_kv_heads=8, prefix_len=512, n_branches=8, gamma=59,
+                    private_len=8192 - 512, vocab=152064, logit_sigma=3.0)
+TREE_DEPTH = 6
+# sources whose change invalidates the DRAM traffic figure kept beside the profile summaries
+KERNEL_SOURCES = ["attn_umma_t.cu", "attn_plan.cuh", "umma_ptx.cuh", "tts_internal.cuh"]
 
 
 def measured_peaks():
     p = ROOT / "MEASURED_PEAKS.json"
     if p.exists():
         d = json.loads(p.read_text())
-        return float(d["hbm_gbs"]), "measured"
-    return FALLBACK_HBM_GBS, "fallback"
+        return float(d["hbm_gbs"]), float(d.get("bf16_tflops_sustained", FALLBACK_BF16_TFLOPS)), "measured"
+    return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback"
+
+
+def kernel_source_hash() -> str:
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        h.update((ROOT / "paper_2505_19634_b200" / "csrc" / name).read_bytes())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(workload: str):
+    """DRAM read + write bytes per launch of the dominant kernel from the last ncu capture, or None when
+    the kernel's sources have changed since (the record carries their hash)."""
+    p = ROOT / "profiles" / "attn_umma_t_kernel_traffic.json"
+    if not p.exists():
+        return None
+    d = json.loads(p.read_text())
+    if d.get("workload") != workload or d.get("kernel_source_hash") != kernel_source_hash():
+        return None
+    return float(d["dram_bytes_per_launch"])
 
 
 def accept_algorithmic_bytes(acc_len: np.ndarray, gamma: int, vocab: int) -> int:
@@ -97,6 +134,30 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def tree_parents_of(shape, seed):
+    return ti.make_tree_parents(shape.n_branches, shape.rows_per_branch, TREE_DEPTH, seed) if shape.name == "tree" else None
+
+
+def tree_flops(shape, parents) -> int:
+    """4*D flops per (query row, visible key): every node sees the prefix, the committed private tokens,
+    itself and its ancestors."""
+    n = shape.rows_per_branch
+    depth = np.zeros(parents.shape, np.int64)
+    for i in range(n):
+        depth[:, i] = np.where(parents[:, i] < 0, 1, depth[np.arange(parents.shape[0]), np.maximum(parents[:, i], 0)] + 1)
+    visible = (shape.prefix_len + shape.lens().astype(np.int64)[:, None] - n) + depth      # [N][n]
+    return int(4 * shape.head_dim * shape.n_q_heads * visible.sum())
+
+
+def oracle_attn(case, shape, parents):
+    import oracle
+    if parents is None:
+        return oracle.verify_attn(case.q, case.k_pages, case.v_pages, case.block_table, case.prefix_len,
+                                  case.branch_lens, shape.gamma)
+    return oracle.verify_attn(case.q, case.k_pages, case.v_pages, case.block_table, case.prefix_len,
+                              case.branch_lens, shape.gamma, mask_kind=1, tree_parents=parents)
+
+
 def oracle_sample(shape: ti.AttnShape, seed: int, budget_s: float = 12.0):
     """Times the CPU oracle on whole layers of the workload (as many passes over one generated
     layer as fit the budget, at most n_layers) plus one accept pass.
@@ -106,20 +167,23 @@ def oracle_sample(shape: ti.AttnShape, seed: int, budget_s: float = 12.0):
     oracle.build()
     bytes_done, secs, layers = 0, 0.0, 0
     case = ti.make_attn_case(shape, seed)
+    parents = tree_parents_of(shape, seed)
     while layers < shape.n_layers:
         t0 = time.perf_counter()
-        oracle.verify_attn(case.q, case.k_pages, case.v_pages, case.block_table, case.prefix_len,
-                           case.branch_lens, shape.gamma)
+        oracle_attn(case, shape, parents)
         dt = time.perf_counter() - t0
         secs += dt; layers += 1; bytes_done += shape.unique_kv_bytes()
         if secs + dt > budget_s:
             break
-    acc_case = ti.make_accept_case(shape.n_branches, shape.gamma, shape.vocab, shape.logit_sigma, seed + 2)
-    t0 = time.perf_counter()
-    acc, _, _ = oracle.accept(acc_case.p_target, acc_case.q_draft, acc_case.draft_tokens, acc_case.uniforms)
-    secs += time.perf_counter() - t0
-    bytes_done += accept_algorithmic_bytes(acc, shape.gamma, shape.vocab)
-    return bytes_done, secs, f"{layers} of {shape.n_layers} layers of attention + 1 accept pass", cores
+    what = f"{layers} of {shape.n_layers} layers of attention"
+    if parents is None:
+        acc_case = ti.make_accept_case(shape.n_branches, shape.gamma, shape.vocab, shape.logit_sigma, seed + 2)
+        t0 = time.perf_counter()
+        acc, _, _ = oracle.accept(acc_case.p_target, acc_case.q_draft, acc_case.draft_tokens, acc_case.uniforms)
+        secs += time.perf_counter() - t0
+        bytes_done += accept_algorithmic_bytes(acc, shape.gamma, shape.vocab)
+        what += " + 1 accept pass"
+    return bytes_done, secs, what, cores
 
 
 def run_reference(args, shape):
@@ -131,11 +195,14 @@ def run_reference(args, shape):
     oracle.build()
     cores = oracle.n_cores()
     case = ti.make_attn_case(shape, 0x5EED + 2)
-    acc_case = ti.make_accept_case(shape.n_branches, shape.gamma, shape.vocab, shape.logit_sigma, 0x5EED + 4)
+    parents = tree_parents_of(shape, 0x5EED + 2)
+    acc_case = None if parents is not None else ti.make_accept_case(shape.n_branches, shape.gamma, shape.vocab,
+                                                                    shape.logit_sigma, 0x5EED + 4)
 
     def step():
-        oracle.verify_attn(case.q, case.k_pages, case.v_pages, case.block_table, case.prefix_len,
-                           case.branch_lens, shape.gamma)
+        oracle_attn(case, shape, parents)
+        if acc_case is None:
+            return None
         a, _, _ = oracle.accept(acc_case.p_target, acc_case.q_draft, acc_case.draft_tokens, acc_case.uniforms)
         return a
     for _ in range(args.warmup):
@@ -144,9 +211,9 @@ def run_reference(args, shape):
     for _ in range(args.steps):
         acc = step()
     dt = (time.perf_counter() - t0) / args.steps
-    nbytes = shape.unique_kv_bytes() + accept_algorithmic_bytes(acc, shape.gamma, shape.vocab)
+    nbytes = shape.unique_kv_bytes() + (accept_algorithmic_bytes(acc, shape.gamma, shape.vocab) if acc is not None else 0)
     gbs = nbytes / dt / 1e9
-    sample = "1 layer of attention + 1 accept pass per step (of %d layers)" % shape.n_layers
+    sample = "1 layer of attention%s per step (of %d layers)" % ("" if acc is None else " + 1 accept pass", shape.n_layers)
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
@@ -159,9 +226,11 @@ def run_reference(args, shape):
 
 
 def workload_name(shape):
+    lens = (f"{shape.n_branches} branches x {shape.private_len} private tokens" if shape.branch_lens is None else
+            f"{shape.n_branches} branches x ragged private tokens {min(shape.branch_lens)}..{max(shape.branch_lens)}")
+    rows = f"{shape.rows_per_branch}-node draft trees (depth <= {TREE_DEPTH})" if shape.name == "tree" else f"gamma={shape.gamma}"
     return (f"{shape.name}-shaped: {shape.n_layers} layers, Hq={shape.n_q_heads}, Hkv={shape.n_kv_heads}, D=128, "
-            f"prefix {shape.prefix_len} + {shape.n_branches} branches x {shape.private_len} private tokens, "
-            f"gamma={shape.gamma}, page 16 (random permutation), vocab {shape.vocab}")
+            f"prefix {shape.prefix_len} + {lens}, {rows}, page 16 (random permutation), vocab {shape.vocab}")
 
 
 def aggregate_over_ranks(ms: float, e2e_ms: float, launches: int, world: int, device):
@@ -179,10 +248,99 @@ def aggregate_over_ranks(ms: float, e2e_ms: float, launches: int, world: int, de
     return float(t[0]), float(t[1]), int(lt[0])
 
 
+class DeviceStep:
+    """The device-resident inputs of one workload and its step (plan + attention per layer [+ accept])."""
+
+    def __init__(self, shape, seed, dev, stream, with_accept=True, first_layer_case=None, parents=None):
+        import torch
+        import paper_2505_19634_b200 as tts
+        self.tts, self.torch, self.shape = tts, torch, shape
+        L, N, V = shape.n_layers, shape.n_branches, shape.vocab
+        self.R = shape.rows_per_branch
+        bt_np, num_pages, max_blocks = ti.make_block_table(shape, seed)
+        self.bt_np, self.lens_np = bt_np, shape.lens()
+        gen = torch.Generator(device=dev); gen.manual_seed(seed)
+        # K/V pools: one per layer, N(0,1) bf16 drawn on the device (Philox); q likewise.  Layer 0 may come from
+        # a host-generated case (the one the oracle checks).
+        pool = lambda: torch.randn(num_pages, shape.n_kv_heads, 16, 128, device=dev, dtype=torch.bfloat16, generator=gen)
+        self.k_pools = [pool() for _ in range(L)]
+        self.v_pools = [pool() for _ in range(L)]
+        self.q_all = torch.randn(L, N, self.R, shape.n_q_heads, 128, device=dev, dtype=torch.bfloat16, generator=gen)
+        if first_layer_case is not None:
+            as_bf16 = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev).view(torch.bfloat16)
+            self.k_pools[0].copy_(as_bf16(first_layer_case.k_pages)); self.v_pools[0].copy_(as_bf16(first_layer_case.v_pages))
+            self.q_all[0].copy_(as_bf16(first_layer_case.q))
+        self.out_all = torch.empty_like(self.q_all)
+        self.bt, self.lens = torch.from_numpy(bt_np).to(dev), torch.from_numpy(self.lens_np).to(dev)
+        self.parents = None if parents is None else torch.from_numpy(np.ascontiguousarray(parents, dtype=np.int32)).to(dev)
+        self.with_accept = with_accept and parents is None
+        if self.with_accept:
+            self.acc_case = ti.make_accept_case(N, shape.gamma, V, shape.logit_sigma, seed + 2)
+            c = self.acc_case
+            self.p_t, self.q_d = torch.from_numpy(c.p_target).to(dev), torch.from_numpy(c.q_draft).to(dev)
+            self.toks, self.unis = torch.from_numpy(c.draft_tokens).to(dev), torch.from_numpy(c.uniforms).to(dev)
+            self.acc_len = torch.zeros(N, dtype=torch.int32, device=dev)
+            self.nxt = torch.zeros(N, dtype=torch.int32, device=dev)
+        self.ctx = tts.TtsContext(shape.n_q_heads, shape.n_kv_heads, N, self.R, max_blocks, num_pages, stream=stream)
+        self.stream = stream
+
+    def step(self, accept=True):
+        s, c, tts = self.shape, self.ctx, self.tts
+        c.tts_attn_plan(self.bt, s.prefix_len, self.lens, s.n_branches, self.R)
+        for l in range(s.n_layers):
+            if self.parents is None:
+                c.tts_verify_attn(self.q_all[l], self.k_pools[l], self.v_pools[l], self.bt, s.prefix_len, self.lens,
+                                  s.n_branches, s.gamma, tts.MASK_CAUSAL, self.out_all[l])
+            else:
+                c.tts_verify_attn_tree(self.q_all[l], self.k_pools[l], self.v_pools[l], self.bt, s.prefix_len,
+                                       self.lens, self.parents, s.n_branches, self.R, self.out_all[l])
+        if self.with_accept and accept:
+            c.tts_accept(self.p_t, self.q_d, self.toks, self.unis, s.n_branches, s.gamma, s.vocab, self.acc_len, self.nxt)
+
+    def capture(self, accept=True):
+        torch = self.torch
+        n0 = self.ctx.tts_launch_count()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=self.stream):
+            self.step(accept)
+        return graph, self.ctx.tts_launch_count() - n0
+
+    def kernel_times_stream(self):
+        """(main us, merge us, launches timed) from CUDA events around the single stream launches of one step:
+        each figure includes the gap of a stream launch, which a graph replay does not pay."""
+        self.ctx.tts_profile_enable(True)
+        self.step()
+        main_us, merge_us, n = self.ctx.tts_profile_read()
+        self.ctx.tts_profile_enable(False)
+        return main_us, merge_us, n
+
+    def out_layer0(self):
+        return self.out_all[0].float().cpu().numpy().astype(np.float64)
+
+
+def time_replays(torch, run, steps, stream, barrier):
+    """K replays between two barriers; an event after every replay gives the per-step times."""
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    barrier()
+    ev[0].record(stream)
+    for i in range(steps):
+        run()
+        ev[i + 1].record(stream)
+    barrier()
+    per = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(steps)])
+    return ev[0].elapsed_time(ev[steps]) / steps, per
+
+
+def attn_errors(got, want):
+    diff = np.abs(got - want)
+    excess = float((diff - (1e-2 + 1e-2 * np.abs(want))).max())
+    rms = float(np.sqrt((diff ** 2).mean()) / max(np.sqrt((want ** 2).mean()), 1e-30))
+    return excess, rms
+
+
 def run_ours(args, shape):
     import torch
     import torch.distributed as dist
-    import paper_2505_19634_b200 as tts
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -195,34 +353,12 @@ def run_ours(args, shape):
     dev = torch.device("cuda", local)
 
     L, N, g, V = shape.n_layers, shape.n_branches, shape.gamma, shape.vocab
-    R = g + 1
     seed = 0x5EED + 2 + 7919 * rank
-    bt_np, num_pages, max_blocks = ti.make_block_table(shape, seed)
-    lens_np = shape.lens()
-    gen = torch.Generator(device=dev); gen.manual_seed(seed)
-    # K/V pools: one per layer, N(0,1) bf16 drawn on the device (Philox); q likewise
-    k_pools = [torch.randn(num_pages, shape.n_kv_heads, 16, 128, device=dev, dtype=torch.bfloat16, generator=gen)
-               for _ in range(L)]
-    v_pools = [torch.randn(num_pages, shape.n_kv_heads, 16, 128, device=dev, dtype=torch.bfloat16, generator=gen)
-               for _ in range(L)]
-    q_all = torch.randn(L, N, R, shape.n_q_heads, 128, device=dev, dtype=torch.bfloat16, generator=gen)
-    out_all = torch.empty_like(q_all)
-    bt, lens = torch.from_numpy(bt_np).to(dev), torch.from_numpy(lens_np).to(dev)
-    acc_case = ti.make_accept_case(N, g, V, shape.logit_sigma, seed + 2)
-    p_t, q_d = torch.from_numpy(acc_case.p_target).to(dev), torch.from_numpy(acc_case.q_draft).to(dev)
-    toks, unis = torch.from_numpy(acc_case.draft_tokens).to(dev), torch.from_numpy(acc_case.uniforms).to(dev)
-    acc_len = torch.zeros(N, dtype=torch.int32, device=dev)
-    nxt = torch.zeros(N, dtype=torch.int32, device=dev)
-
+    parents = tree_parents_of(shape, seed)
     stream = torch.cuda.Stream(device=dev)      # a side stream: graph capture needs one
     torch.cuda.set_stream(stream)
-    ctx = tts.TtsContext(shape.n_q_heads, shape.n_kv_heads, N, R, max_blocks, num_pages, stream=stream)
-
-    def step():
-        for l in range(L):
-            ctx.tts_verify_attn(q_all[l], k_pools[l], v_pools[l], bt, shape.prefix_len, lens, N, g,
-                                tts.MASK_CAUSAL, out_all[l])
-        ctx.tts_accept(p_t, q_d, toks, unis, N, g, V, acc_len, nxt)
+    ds = DeviceStep(shape, seed, dev, stream, parents=parents)
+    ctx = ds.ctx
 
     def barrier():
         torch.cuda.synchronize()
@@ -231,17 +367,13 @@ def run_ours(args, shape):
             torch.cuda.synchronize()
 
     for _ in range(max(args.warmup, 3)):
-        step()
+        ds.step()
     barrier()
-    # The library's calls of one step (64 x attention + accept) are captured once into a CUDA graph and
-    # the timed steps replay it: the same kernels on the same arguments, without the per-launch gaps.
-    graph, run_step, launches_per_step = None, step, None
+    # The library's calls of one step are captured once into a CUDA graph and the timed steps replay it:
+    # the same kernels on the same arguments, without the per-launch gaps.
+    graph, run_step, launches_per_step = None, ds.step, None
     if not args.no_graph:
-        n0 = ctx.tts_launch_count()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=stream):
-            step()
-        launches_per_step = ctx.tts_launch_count() - n0
+        graph, launches_per_step = ds.capture()
         run_step = graph.replay
         for _ in range(3):
             run_step()
@@ -250,85 +382,105 @@ def run_ours(args, shape):
     if rank == 0:
         sampler.start()
     launches0 = ctx.tts_launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record(stream)
-    for _ in range(args.steps):
-        run_step()
-    e1.record(stream)
-    barrier()
-    ms = e0.elapsed_time(e1) / args.steps
+    ms, per_step = time_replays(torch, run_step, args.steps, stream, barrier)
     launches = launches_per_step * args.steps if graph is not None else ctx.tts_launch_count() - launches0
     status = ctx.tts_last_status()
     if status != 0:
         raise SystemExit(f"device status {status} after the timed region")
 
-    # dominant kernel alone: the attention main kernel, event-timed per launch over K more steps
-    ctx.tts_profile_enable(True)
-    for _ in range(min(args.steps, 4096 // L)):
-        step()
-    main_us, merge_us, prof_calls = ctx.tts_profile_read()
-    ctx.tts_profile_enable(False)
+    # The dominant kernel in the launch mode of the timed steps: a graph of the attention calls alone (schedule +
+    # per layer the main kernel and its merge kernel), timed like the step.  Its time per layer bounds the main
+    # kernel's duration from above (an event between two kernel nodes of a graph would add its own latency).
+    if graph is not None:
+        attn_graph, _ = ds.capture(accept=False)
+        for _ in range(3):
+            attn_graph.replay()
+        attn_ms, _ = time_replays(torch, attn_graph.replay, args.steps, stream, barrier)
+        del attn_graph
+    else:
+        attn_ms, _ = time_replays(torch, lambda: ds.step(accept=False), args.steps, stream, barrier)
+    layer_us = attn_ms * 1e3 / L
+    main_us, merge_us, prof_calls = ds.kernel_times_stream()
     clocks = sampler.stop() if rank == 0 else None
 
-    acc_host = acc_len.cpu().numpy()
-    step_bytes = shape.unique_kv_bytes() * L + accept_algorithmic_bytes(acc_host, g, V)
+    acc_bytes = accept_algorithmic_bytes(ds.acc_len.cpu().numpy(), g, V) if ds.with_accept else 0
+    step_bytes = shape.unique_kv_bytes() * L + acc_bytes
 
-    # ---- end to end through the host entry point ----
-    q_host = torch.empty(q_all.shape, dtype=torch.bfloat16, pin_memory=True); q_host.copy_(q_all)
-    out_host = torch.empty(q_all.shape, dtype=torch.bfloat16, pin_memory=True)
-    pin = lambda a: torch.from_numpy(a).pin_memory()
-    h_bt, h_lens = pin(bt_np), pin(lens_np)
-    h_p, h_q, h_t, h_u = pin(acc_case.p_target), pin(acc_case.q_draft), pin(acc_case.draft_tokens), pin(acc_case.uniforms)
-    h_al = torch.zeros(N, dtype=torch.int32).pin_memory(); h_nt = torch.zeros(N, dtype=torch.int32).pin_memory()
+    # ---- end to end through the host entry point (chains only) ----
+    e2e = None
+    if ds.with_accept:
+        q_host = torch.empty(ds.q_all.shape, dtype=torch.bfloat16, pin_memory=True); q_host.copy_(ds.q_all)
+        out_host = torch.empty(ds.q_all.shape, dtype=torch.bfloat16, pin_memory=True)
+        pin = lambda a: torch.from_numpy(a).pin_memory()
+        c = ds.acc_case
+        h_bt, h_lens = pin(ds.bt_np), pin(ds.lens_np)
+        h_p, h_q, h_t, h_u = pin(c.p_target), pin(c.q_draft), pin(c.draft_tokens), pin(c.uniforms)
+        h_al = torch.zeros(N, dtype=torch.int32).pin_memory(); h_nt = torch.zeros(N, dtype=torch.int32).pin_memory()
 
-    def step_host():
-        ctx.tts_verify_step_host(L, q_host, k_pools, v_pools, h_bt, shape.prefix_len, h_lens, N, g, h_p, h_q, h_t,
-                                 h_u, V, out_host, h_al, h_nt)
-    e2e_steps = max(2, min(args.steps, 5))
-    for _ in range(2):
-        step_host()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        step_host()
-    torch.cuda.synchronize()
-    e2e_ms = (time.perf_counter() - t0) / e2e_steps * 1e3
-    h2d = (q_host.numel() * 2 + h_bt.numel() * 4 + h_lens.numel() * 4 + h_p.numel() * 4 + h_q.numel() * 4 +
-           h_t.numel() * 4 + h_u.numel() * 4)
-    d2h = out_host.numel() * 2 + 8 * N
+        def step_host():
+            ctx.tts_verify_step_host(L, q_host, ds.k_pools, ds.v_pools, h_bt, shape.prefix_len, h_lens, N, g, h_p, h_q,
+                                     h_t, h_u, V, out_host, h_al, h_nt)
+        e2e_steps = max(2, min(args.steps, 5))
+        for _ in range(2):
+            step_host()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            step_host()
+        torch.cuda.synchronize()
+        e2e_ms = (time.perf_counter() - t0) / e2e_steps * 1e3
+        h2d = (q_host.numel() * 2 + h_bt.numel() * 4 + h_lens.numel() * 4 + h_p.numel() * 4 + h_q.numel() * 4 +
+               h_t.numel() * 4 + h_u.numel() * 4)
+        d2h = out_host.numel() * 2 + 8 * N
+    else:
+        e2e_ms, h2d, d2h = 0.0, 0, 0
 
     ms, e2e_ms, launches = aggregate_over_ranks(ms, e2e_ms, launches, world, dev)
 
     if rank == 0:
-        peak, peak_kind = measured_peaks()
+        peak, tf_peak, peak_kind = measured_peaks()
         total_bytes = step_bytes * world
         value = total_bytes / (ms * 1e-3) / 1e9
         layer_bytes = shape.unique_kv_bytes()
-        # DRAM read + write bytes of one launch of the dominant kernel, from the ncu capture summarised in
-        # profiles/attn_umma_t_kernel_32b_2layers.md (valid for the 32b workload and this kernel version only)
-        traffic = 276.4e6 if shape.name == "32b" else None
-        roof = {"bound": "hbm", "achieved": None, "peak": peak, "unit": "GB/s", "frac": None, "traffic": traffic,
-                "peak_kind": f"of {peak_kind}", "kernel": "attn_umma_t_kernel (token-major tcgen05 attention, one layer per launch)"}
-        if main_us:
-            roof["achieved"] = layer_bytes / (main_us * 1e-6) / 1e9
+        is_tree = parents is not None
+        kernel = ("attn_umma_kernel (row-major tcgen05 attention, one layer per launch)" if is_tree else
+                  "attn_umma_t_kernel (token-major tcgen05 attention, one layer per launch)")
+        if is_tree:
+            flops = tree_flops(shape, parents)
+        timing = ("duration = time per layer of a %s of the attention calls alone (main kernel + merge kernel), CUDA events "
+                  "around %d replays: an upper bound for the main kernel, so achieved and frac are lower bounds"
+                  % ("graph replay" if graph is not None else "stream-launched run", args.steps))
+        if is_tree:
+            flops = tree_flops(shape, parents)
+            roof = {"bound": "tensor", "achieved": flops / (layer_us * 1e-6) / 1e12, "peak": tf_peak, "unit": "TFLOP/s",
+                    "traffic": None, "peak_kind": f"of {peak_kind} (sustained bf16 GEMM)", "kernel": kernel,
+                    "flops_per_launch": flops}
+            roof["frac"] = roof["achieved"] / tf_peak
+        else:
+            roof = {"bound": "hbm", "achieved": layer_bytes / (layer_us * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
+                    "traffic": recorded_traffic(shape.name) if not args.layers else None,
+                    "peak_kind": f"of {peak_kind}", "kernel": kernel, "algorithmic_bytes_per_launch": layer_bytes}
             roof["frac"] = roof["achieved"] / peak
-            roof["kernel_us"] = main_us
-            roof["merge_kernel_us"] = merge_us
-            roof["launches_timed"] = prof_calls
+            roof["frac_of_nominal_peak"] = roof["achieved"] / NOMINAL_HBM_GBS
+        roof.update({"kernel_us": layer_us, "kernel_timing": timing,
+                     "stream_launch_events": {"main_kernel_us": main_us, "merge_kernel_us": merge_us, "launches": prof_calls,
+                                              "note": "CUDA events around single stream launches; each includes the launch gap"}})
         cb_bytes, cb_s, cb_sample, cores = oracle_sample(shape, 0x5EED + 2)
         rec = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "ms_per_step_median": float(np.median(per_step)), "ms_per_step_min": float(per_step.min()),
             "us_per_layer": ms * 1e3 / L,
-            "frac_of_hbm_peak": value / world / peak,
+            "frac_of_measured_peak": value / world / peak, "measured_peak_gbs": peak,
+            "frac_of_nominal_peak": value / world / NOMINAL_HBM_GBS, "nominal_peak_gbs": NOMINAL_HBM_GBS,
             "config": {"workload": workload_name(shape), "l2": "inputs larger than L2: %.2f GiB of KV per step, one K/V pool per layer (for a one-layer "
                              "config: that many independent copies of the layer)" % (layer_bytes * L / 2**30), "bytes_per_step": step_bytes,
                        "launch": "one CUDA graph replay per step" if graph is not None else "stream launches",
+                       "step": "tts_attn_plan + %d x attention%s" % (L, " + tts_accept" if ds.with_accept else ""),
                        "attn_impl": "auto"},
             "clocks": clocks,
-            "e2e": {"value": total_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
+            "e2e": {"value": total_bytes / (e2e_ms * 1e-3) / 1e9 if e2e_ms else None, "unit": "GB/s", "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": launches,
             "roofline": roof,
@@ -341,25 +493,94 @@ def run_ours(args, shape):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """The branch / draft-length sweep on the 32B layer shape: every point timed L2-cold (a rotation over
+    enough independent copies of the layer) and checked against the oracle (all rows of the first copy)."""
+    import torch
+    import oracle
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    stream = torch.cuda.Stream(device=dev)
+    torch.cuda.set_stream(stream)
+    peak, _, peak_kind = measured_peaks()
+    oracle.build()
+    rows, worst_excess, worst_rms = [], -1.0, 0.0
+    print("| N | gamma | seed | private tokens | prefix | unique KV MB | layers rotated | us/layer | GB/s | frac of %s peak | max excess over band | rel RMS err |" % peak_kind)
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|")
+    for n in ti.SWEEP_BRANCHES:
+        for g in ti.SWEEP_GAMMAS:
+            for seed in range(args.seeds):
+                shp = ti.sweep_shape(n, g, 1000 * seed + 10 * n + g)
+                copies = max(2, -(-2 * L2_BYTES // shp.unique_kv_bytes()))
+                shp = replace(shp, n_layers=copies)
+                case = ti.make_attn_case(shp, 77 + seed)
+                ti.poison_unused_slots(case)
+                ds = DeviceStep(shp, 77 + seed, dev, stream, with_accept=False, first_layer_case=case)
+                for _ in range(3):
+                    ds.step()
+                torch.cuda.synchronize()
+                excess, rms = attn_errors(ds.out_layer0(), oracle_attn(case, shp, None))
+                graph, _ = ds.capture()
+                for _ in range(3):
+                    graph.replay()
+                ms, _ = time_replays(torch, graph.replay, args.steps, stream, torch.cuda.synchronize)
+                status = ds.ctx.tts_last_status()
+                us = ms * 1e3 / copies
+                gbs = shp.unique_kv_bytes() / us / 1e3
+                worst_excess, worst_rms = max(worst_excess, excess), max(worst_rms, rms)
+                rows.append(dict(N=n, gamma=g, seed=seed, us_per_layer=us, gbs=gbs, frac=gbs / peak, excess=excess, rms=rms,
+                                 status=status))
+                print(f"| {n} | {g} | {seed} | {int(shp.lens().sum())} | {shp.prefix_len} | {shp.unique_kv_bytes() / 1e6:.1f} | {copies} | "
+                      f"{us:.2f} | {gbs:.0f} | {gbs / peak:.3f} | {excess:+.2e} | {rms:.2e} |", flush=True)
+                del graph
+                ds.ctx.close()
+                del ds
+                torch.cuda.empty_cache()
+    ok = worst_excess <= 0 and worst_rms <= 5e-3 and all(r["status"] == 0 for r in rows)
+    best = max(rows, key=lambda r: r["gbs"])
+    print(json.dumps({"metric": METRIC, "value": best["gbs"], "unit": "GB/s", "n_gpus": 1, "steps": args.steps, "warmup": 3,
+                      "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": "sweep on the 32B layer shape: N in %s x gamma in %s x %d seeds, ragged private lengths "
+                                 "1024..8192, prefix 256..1024, random page permutation; L2-cold rotation over copies of the layer; "
+                                 "value = the best point" % (list(ti.SWEEP_BRANCHES), list(ti.SWEEP_GAMMAS), args.seeds)},
+                      "parity": {"points": len(rows), "all_inside_band": ok, "worst_excess_over_band": worst_excess,
+                                 "worst_rel_rms": worst_rms},
+                      "points": rows}, ensure_ascii=False))
+    if not ok:
+        raise SystemExit("sweep: a point left the oracle's band")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="32b", choices=list(ti.CONFIGS))
+    ap.add_argument("--config", default="32b", choices=list(ti.CONFIGS) + ["tree", "sweep"])
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA graph replay")
     ap.add_argument("--layers", type=int, default=0,
                     help="run only this many layers of the config (small cases for profiler captures; "
                          "the workload name says so)")
+    ap.add_argument("--seeds", type=int, default=3, help="seeds per point of --config sweep")
+    ap.add_argument("--kernel-hash", action="store_true", help="print the hash of the dominant kernel's sources and exit")
     args = ap.parse_args()
-    shape = ti.CONFIGS[args.config]
+    if args.kernel_hash:
+        print(kernel_source_hash())
+        return
+    if args.config == "sweep":
+        if args.impl == "reference":
+            raise SystemExit("the sweep has no reference arm (every point is checked against the oracle inside the run)")
+        run_sweep(args)
+        return
+    shape = TREE if args.config == "tree" else ti.CONFIGS[args.config]
     if args.layers > 0:
-        shape = ti.with_branches(shape, n_layers=args.layers)
+        shape = replace(shape, n_layers=args.layers)
     elif shape.n_layers == 1:
-        # a one-layer config fits L2 (126 MB): time a rotation over enough independent copies of the
+        # a one-layer config fits L2 (126 MB) or nearly: time a rotation over enough independent copies of the
         # layer (own K/V/Q each) that the working set exceeds twice the L2
-        shape = ti.with_branches(shape, n_layers=-(-2 * 132_000_000 // shape.unique_kv_bytes()))
+        shape = replace(shape, n_layers=max(2, -(-2 * L2_BYTES // shape.unique_kv_bytes())))
     if args.impl == "reference":
         run_reference(args, shape)
     else:

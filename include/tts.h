@@ -252,7 +252,9 @@ TTS_API int64_t tts_launch_count(tts_ctx* ctx);
  * before its main kernel, between the main kernel and the merge kernel, and after the merge (at
  * most 4096 calls are kept).  tts_profile_read synchronises the stream, writes the mean duration
  * in microseconds of the main kernel and of the merge kernel over the recorded calls and their
- * number (host pointers), and forgets them.
+ * number (host pointers), and forgets them.  Calls made while the stream is being captured into a
+ * CUDA graph put the events into the graph: read after a replay, the durations are those of the
+ * kernels inside that replay (without the gap that a stream launch adds between two events).
  */
 TTS_API int tts_profile_enable(tts_ctx* ctx, int on);
 TTS_API int tts_profile_read(tts_ctx* ctx, float* attn_main_us, float* attn_merge_us, int* n_calls);

@@ -53,21 +53,36 @@ __device__ __forceinline__ void draw_token(const float* __restrict__ pk, const f
     for (int attempt = 0; attempt < 2; ++attempt) {
         // ---- 2. one sweep: per-tile fp64 sums ----
         int last_pos = -1;
-        for (int j = warp; j < n_tiles; j += kAccThreads / 32) {
-            const int x0 = j * kTileElems + lane * 4;
-            double s = 0.0;
-            if (x0 < vocab) {                                   // vocab % 4 == 0: whole float4 in range
-                const float4 pv = __ldg(reinterpret_cast<const float4*>(pk + x0));
-                float4 qv = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (residual) qv = __ldg(reinterpret_cast<const float4*>(qk + x0));
-                const float w0 = weight(pv.x, qv.x, residual), w1 = weight(pv.y, qv.y, residual);
-                const float w2 = weight(pv.z, qv.z, residual), w3 = weight(pv.w, qv.w, residual);
-                s = (double)w0 + (double)w1 + (double)w2 + (double)w3;
-                if (w3 > 0.f) last_pos = x0 + 3; else if (w2 > 0.f) last_pos = x0 + 2;
-                else if (w1 > 0.f) last_pos = x0 + 1; else if (w0 > 0.f) last_pos = x0;
+        // kSweepBatch tiles per warp and trip: their loads are all issued before the first is used (one SM has
+        // to keep many loads in flight to pull its share of the bandwidth)
+        constexpr int kSweepBatch = 4, kWarps = kAccThreads / 32;
+        for (int j0 = warp; j0 < n_tiles; j0 += kWarps * kSweepBatch) {
+            float4 pv[kSweepBatch], qv[kSweepBatch];
+#pragma unroll
+            for (int k = 0; k < kSweepBatch; ++k) {
+                const int x0 = (j0 + k * kWarps) * kTileElems + lane * 4;
+                pv[k] = qv[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (j0 + k * kWarps < n_tiles && x0 < vocab) {      // vocab % 4 == 0: whole float4 in range
+                    pv[k] = __ldg(reinterpret_cast<const float4*>(pk + x0));
+                    if (residual) qv[k] = __ldg(reinterpret_cast<const float4*>(qk + x0));
+                }
             }
-            s = warp_sum(s);
-            if (lane == 0) tile_sum[j] = s;
+#pragma unroll
+            for (int k = 0; k < kSweepBatch; ++k) {
+                const int j = j0 + k * kWarps;
+                if (j >= n_tiles) break;                            // uniform over the warp
+                const int x0 = j * kTileElems + lane * 4;
+                double s = 0.0;
+                if (x0 < vocab) {
+                    const float w0 = weight(pv[k].x, qv[k].x, residual), w1 = weight(pv[k].y, qv[k].y, residual);
+                    const float w2 = weight(pv[k].z, qv[k].z, residual), w3 = weight(pv[k].w, qv[k].w, residual);
+                    s = (double)w0 + (double)w1 + (double)w2 + (double)w3;
+                    if (w3 > 0.f) last_pos = max(last_pos, x0 + 3); else if (w2 > 0.f) last_pos = max(last_pos, x0 + 2);
+                    else if (w1 > 0.f) last_pos = max(last_pos, x0 + 1); else if (w0 > 0.f) last_pos = max(last_pos, x0);
+                }
+                s = warp_sum(s);
+                if (lane == 0) tile_sum[j] = s;
+            }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xffffffffu, last_pos, o));

@@ -11,12 +11,16 @@ namespace {
 
 constexpr int kPlanThreads = 1024;
 
+// Where the pages of one of a CTA's first two tiles are listed: block-table row, first block, number of
+// pages, KV head (-1 pages: no such tile).
+struct FirstTile { int bt_row, blk0, n_pages, kvh; };
+
 // Walks the run of CTA c.  With out == nullptr only counts its pieces.
-__device__ int walk_run(const AttnParams& p, const int* cum, int total, int tpc, int c, PieceDesc* out, CtaPlan* hdr) {
+__device__ int walk_run(const AttnParams& p, const int* cum, int total, int tpc, int c, PieceDesc* out, CtaPlan* hdr, FirstTile* first2) {
     const int g_begin = c * tpc, g_end = min(total, g_begin + tpc);
     if (hdr) {
         hdr->n_tiles = max(0, g_end - g_begin);
-        for (int i = 0; i < 16; ++i) hdr->first_pages[i] = -1;
+        first2[0].n_pages = first2[1].n_pages = 0;
     }
     if (g_begin >= g_end) return 0;
     SegInfo seg = segment_of_tile(p, cum, g_begin);
@@ -35,12 +39,11 @@ __device__ int walk_run(const AttnParams& p, const int* cum, int total, int tpc,
             d.pad = 0;
             out[n] = d;
             if (n < kPlanInline) hdr->first_pieces[n] = d;
-            const int32_t* bt = p.block_table + (size_t)d.bt_row * p.max_blocks;
             for (int t = t_first; t < t_last && u < 2; ++t, ++u) {
                 const int tok0 = t * p.tile_tokens;
-                const int n_pages = ceil_div(min(p.tile_tokens, seg.n_tokens - tok0), kPage);
-                for (int j = 0; j < n_pages && j < 8; ++j)
-                    hdr->first_pages[u * 8 + j] = checked_page(p, bt, (seg.tok_begin + tok0) / kPage + j) * p.Hkv + seg.kvh;
+                first2[u].bt_row = d.bt_row; first2[u].blk0 = (seg.tok_begin + tok0) / kPage;
+                first2[u].n_pages = min(8, ceil_div(min(p.tile_tokens, seg.n_tokens - tok0), kPage));
+                first2[u].kvh = seg.kvh;
             }
         }
         ++n;
@@ -54,19 +57,40 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(const AttnParam
     extern __shared__ int sm[];
     int* cum = sm;                                         // N + 1 ints
     int* first = sm + p.N + 1;                             // grid + 1 ints: index of every CTA's first piece
+    FirstTile* first2 = reinterpret_cast<FirstTile*>(first + p.grid + 1);   // 2 per CTA
     build_branch_tile_prefix(p, cum);
     const int total = total_tiles(p, cum);
     const int tpc = ceil_div(total, p.grid);
-    for (int c = threadIdx.x; c < p.grid; c += blockDim.x) first[c + 1] = walk_run(p, cum, total, tpc, c, nullptr, nullptr);
+    for (int c = threadIdx.x; c < p.grid; c += blockDim.x) first[c + 1] = walk_run(p, cum, total, tpc, c, nullptr, nullptr, nullptr);
     __syncthreads();
-    if (threadIdx.x == 0) {                                // a few hundred additions
-        first[0] = 0;
-        for (int c = 0; c < p.grid; ++c) first[c + 1] += first[c];
+    if (threadIdx.x < 32) {                                // inclusive scan of the counts by the first warp, 32 at a time
+        const int lane = threadIdx.x;
+        int carry = 0;
+        for (int base = 0; base < p.grid; base += 32) {
+            int v = base + lane < p.grid ? first[base + lane + 1] : 0;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int n = __shfl_up_sync(0xffffffffu, v, o);
+                if (lane >= o) v += n;
+            }
+            if (base + lane < p.grid) first[base + lane + 1] = carry + v;
+            carry += __shfl_sync(0xffffffffu, v, 31);
+        }
+        if (lane == 0) first[0] = 0;
     }
     __syncthreads();
     for (int c = threadIdx.x; c < p.grid; c += blockDim.x) {
         cta[c].piece_begin = first[c];
-        cta[c].n_pieces = walk_run(p, cum, total, tpc, c, pieces + first[c], cta + c);
+        cta[c].n_pieces = walk_run(p, cum, total, tpc, c, pieces + first[c], cta + c, first2 + 2 * c);
+    }
+    __syncthreads();
+    // the pages of every CTA's first two tiles: one thread per page, all loads independent
+    for (int i = threadIdx.x; i < p.grid * 16; i += blockDim.x) {
+        const int c = i >> 4, j = i & 7;
+        const FirstTile ft = first2[2 * c + ((i >> 3) & 1)];
+        int page_head = -1;
+        if (j < ft.n_pages) page_head = checked_page(p, p.block_table + (size_t)ft.bt_row * p.max_blocks, ft.blk0 + j) * p.Hkv + ft.kvh;
+        cta[c].first_pages[i & 15] = page_head;
     }
     constexpr int kEntries = kMaxPrivBlocks + kMaxPreBlocks;
     if (groups)
@@ -81,7 +105,7 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(const AttnParam
 cudaError_t launch_attn_plan(const AttnParams& main_params, cudaStream_t st) {
     AttnParams p = main_params;
     p.lens_smem = 0;
-    const size_t smem = (size_t)(p.N + 1 + p.grid + 1) * sizeof(int);
+    const size_t smem = (size_t)(p.N + 1 + p.grid + 1) * sizeof(int) + (size_t)p.grid * 2 * sizeof(FirstTile);
     attn_plan_kernel<<<1, kPlanThreads, smem, st>>>(p, const_cast<CtaPlan*>(p.plan_cta), const_cast<PieceDesc*>(p.plan_pieces),
                                                     static_cast<GroupDesc*>(p.group_desc));
     return cudaGetLastError();

@@ -213,12 +213,43 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Abort ab{misc, p.status};
 
-    // ---- set-up: barriers, TMEM, tensor-map prefetch, and this CTA's record of the plan (one coalesced read) ----
+    // ---- first of all, the loads of the CTA's first two tiles: each producer warp sets up the barriers of its
+    // own ring, takes the tiles' pages straight from the plan in global memory and issues the copies; the data
+    // is then on its way while the rest of the set-up runs ----
+    int n_early = 0;                                       // tiles already issued (producer warps)
+    if (warp == kProducerWarp || warp == kProducerWarp + 1) {
+        const int op = warp - kProducerWarp;
+        const int ring0 = op == 0 ? 0 : NK, ring_n = op == 0 ? NK : NV;
+        static_assert(NK >= 2 && NV >= 2, "the first two tiles go to slots 0 and 1 of either ring");
+        if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(op == 0 ? &tm_k : &tm_v) : "memory");
+        int ph = -1;
+        if (lane < 16) ph = __ldg(&p.plan_cta[blockIdx.x].first_pages[lane]);
+        if (lane == 0) {
+            for (int i = 0; i < ring_n; ++i) { mbar_init(bar(L::FULL + ring0 + i), 1); mbar_init(bar(L::EMPTY + ring0 + i), 1); }
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncwarp();
+        const unsigned have = __ballot_sync(0xffffffffu, ph >= 0);
+        const uint64_t stream_once = l2_policy_evict_first();
+        const CUtensorMap* tm = op == 0 ? &tm_k : &tm_v;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int n_pages = __popc((have >> (8 * u)) & 0xffu);      // uniform
+            const int my = __shfl_sync(0xffffffffu, ph, 8 * u + (lane & 7));
+            if (n_pages > 0) {
+                if (lane == 0) mbar_arrive_expect_tx(bar(L::FULL + ring0 + u), (uint32_t)n_pages * 4096u);
+                __syncwarp();
+                if (lane < n_pages)
+                    tma_load_page(sbase + L::kOffRing + (ring0 + u) * kSlotBytes + lane * 4096, tm, my, bar(L::FULL + ring0 + u), stream_once);
+                ++n_early;
+            }
+        }
+    }
+    // ---- set-up: the other barriers, TMEM, tensor-map prefetch, and this CTA's record of the plan (one coalesced read) ----
     if (tid >= 32 && tid < 64)
         reinterpret_cast<uint4*>(smem + L::kOffPlan)[tid - 32] = __ldg(reinterpret_cast<const uint4*>(p.plan_cta + blockIdx.x) + (tid - 32));
     if (tid == 0) {
         misc[0] = 0;
-        for (int i = 0; i < NS; ++i) { mbar_init(bar(L::FULL + i), 1); mbar_init(bar(L::EMPTY + i), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(bar(L::S_FULL + i), 1); mbar_init(bar(L::S_FREE + i), 4 * CG); }
         mbar_init(bar(L::P_FULL), 4 * CG); mbar_init(bar(L::P_FREE), 1);     // softmax warps arrive once per warp
         mbar_init(bar(L::Q_FULL), 4 * CG);
@@ -232,8 +263,6 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + L::kOffMisc + 4), "r"(L::kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    if (warp == kProducerWarp && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
-    if (warp == kProducerWarp + 1 && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
@@ -261,6 +290,10 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
             for (int i = 0; i < pc.n_tiles && alive; ++i, ++u) {
                 const int tok0 = (pc.tile0 + i) * kTileT;
                 const int n_pages = ceil_div(min(kTileT, pc.seg_tokens - tok0), kPage);
+                if (u < n_early) {                             // issued at the start of the kernel
+                    if (++ring_pos == ring_n) { ring_pos = 0; ring_round ^= 1; }
+                    continue;
+                }
                 int page_head = 0;                             // page * Hkv + kvh: the TMA coordinate of a page-head tile
                 if (lane < n_pages)
                     page_head = u < 2 ? rec->first_pages[u * 8 + lane]
@@ -379,13 +412,17 @@ attn_umma_t_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
             alive = __all_sync(0xffffffffu, alive);
             if (!alive) break;
             tc_fence_after();
-            for (int r0 = 0; r0 < n_rows; r0 += 4) {
-                float o[4];
-                tmem_ld4(tmem_o0 + (uint32_t)(pb * NB) + lane_base + (uint32_t)r0, o);
+            {   // all rows of this thread's head dim in one round trip to TMEM, then the stores
+                float o[NB / 4][4];
+#pragma unroll
+                for (int k = 0; k < NB / 4; ++k)
+                    if (4 * k < n_rows) tmem_ld4(tmem_o0 + (uint32_t)(pb * NB) + lane_base + (uint32_t)(4 * k), o[k]);
                 tmem_wait_ld();
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (r0 + e < n_rows) po[(size_t)(r0 + e) * kHeadDim + dim] = o[e];
+                for (int k = 0; k < NB / 4; ++k)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (4 * k + e < n_rows) po[(size_t)(4 * k + e) * kHeadDim + dim] = o[k][e];
             }
             if (et < n_rows) {
                 const float* ls = lsum + pb * 4 * NB + et;

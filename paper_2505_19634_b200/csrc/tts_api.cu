@@ -177,7 +177,14 @@ int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
     }
     const bool prof = c->profiling && c->prof_ev && c->prof_n < kProfMaxCalls;
     cudaEvent_t* ev = prof ? c->prof_ev + 3 * c->prof_n : nullptr;
-    if (prof) cudaEventRecord(ev[0], c->stream);
+    // inside a stream capture the events become event-record nodes of the graph: every replay records them
+    cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
+    if (prof) cudaStreamIsCapturing(c->stream, &capture);
+    auto record = [&](cudaEvent_t event) {
+        if (capture == cudaStreamCaptureStatusActive) cudaEventRecordWithFlags(event, c->stream, cudaEventRecordExternal);
+        else cudaEventRecord(event, c->stream);
+    };
+    if (prof) record(ev[0]);
     if (pl.impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR) {
         e = launch_attn_umma_t(c, p, c->stream);
     } else if (pl.impl == TTS_ATTN_TCGEN05_ROW_MAJOR) {
@@ -188,11 +195,11 @@ int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
     }
     if (e != cudaSuccess) return cuda_fail(c, e);
     c->launches += 1;
-    if (prof) cudaEventRecord(ev[1], c->stream);
+    if (prof) record(ev[1]);
     e = launch_attn_combine(p, c->stream);
     if (e != cudaSuccess) return cuda_fail(c, e);
     c->launches += 1;
-    if (prof) { cudaEventRecord(ev[2], c->stream); c->prof_n += 1; }
+    if (prof) { record(ev[2]); c->prof_n += 1; }
     return TTS_OK;
 }
 
