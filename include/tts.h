@@ -258,6 +258,15 @@ TTS_API int64_t tts_launch_count(tts_ctx* ctx);
  */
 TTS_API int tts_profile_enable(tts_ctx* ctx, int on);
 TTS_API int tts_profile_read(tts_ctx* ctx, float* attn_main_us, float* attn_merge_us, int* n_calls);
+/*
+ * Diagnostics of the failure-detection path.  Every wait inside the tensor-core kernels (on a TMA copy,
+ * on another warp role) is bounded: when its limit runs out the kernel raises TTS_ERR_DEVICE_TIMEOUT in
+ * the device status word, lets go of what it holds and returns, so a lost signal never hangs the GPU.
+ * tts_debug_wait_timeout runs a separate one-warp kernel on the context's stream that waits, through the
+ * same routine, limit_ns nanoseconds (1 us .. 1 s) for a signal that is never sent.  Afterwards
+ * tts_last_status reports TTS_ERR_DEVICE_TIMEOUT and the context works as before.
+ */
+TTS_API int tts_debug_wait_timeout(tts_ctx* ctx, int64_t limit_ns);
 /* Static, NUL-terminated description of a tts_status. */
 TTS_API const char* tts_strerror(int status);
 

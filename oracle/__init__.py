@@ -123,6 +123,31 @@ def accept(p_target, q_draft, draft_tokens, uniforms, n_threads=None):
     return acc, nxt, near
 
 
+def softmax_rows(logits, n_threads=None):
+    """fp32 probabilities from logits [..., V] (fp32, or uint16 bf16 bits, which are widened exactly), by the
+    step-by-step fp32 arithmetic written out above `oracle_softmax_rows` in tts_oracle.cpp."""
+    a = np.asarray(logits)
+    if a.dtype == np.uint16:
+        a = (a.astype(np.uint32) << np.uint32(16)).view(np.float32)
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    out = np.empty_like(a)
+    V = a.shape[-1]
+    rc = lib().oracle_softmax_rows(_p(a, ctypes.c_float), ctypes.c_long(a.size // V), ctypes.c_int(V),
+                                   _p(out, ctypes.c_float), ctypes.c_int(int(n_threads or n_cores())))
+    if rc != 0:
+        raise ValueError("oracle_softmax_rows: inconsistent arguments")
+    return out
+
+
+def accept_logits(target_logits, draft_logits, draft_tokens, uniforms, n_threads=None):
+    """The accept rule fed with logits: p_i = softmax_rows(target_logits[:, i]), q_i = softmax_rows(draft_logits
+    [:, i]), then `accept` on those probabilities, unchanged.  Returns (accepted_len, next_token, near_flags)."""
+    p = softmax_rows(target_logits, n_threads)
+    N, R, V = p.shape
+    q = softmax_rows(draft_logits, n_threads) if R > 1 else np.zeros((N, 0, V), np.float32)
+    return accept(p, q, draft_tokens, uniforms, n_threads)
+
+
 def majority_vote(answers, weights=None, mode: int = 0):
     """Returns (winner, votes, score)."""
     answers = np.ascontiguousarray(answers, dtype=np.int64)

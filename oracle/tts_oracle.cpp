@@ -236,6 +236,57 @@ int oracle_accept(const float* p_target, const float* q_draft, const int32_t* dr
 }
 
 // ---------------------------------------------------------------------------------
+// Probabilities from logits, for the accept rule fed with logits instead of probabilities (the
+// softmax that sits between the target model's last layer and the accept test; Section 2,
+// "Speculative decoding": the rule compares the target's and the draft's token distributions).
+// The paper fixes no arithmetic for it; this is the reading, chosen so that the accept decisions
+// can be reproduced bit for bit: every step is one correctly rounded fp32 operation (or one fp64
+// sum), none of them left to a library exp.
+//   per row l[0..V):  m = max_x l(x)
+//     d = l(x) - m                       fp32 subtract
+//     y = d * log2(e)                    fp32 multiply, log2(e) rounded to fp32
+//     n = round-to-nearest-even(y),  f = y - n   (exact, |f| <= 1/2)
+//     g = c0 + f (c1 + f (c2 + ... f c7))  eight-term Taylor polynomial of 2^f = exp(f ln 2), every
+//                                          step one fp32 fused multiply-add, c_k = (ln 2)^k / k! in fp32
+//     e(x) = g * 2^n   (exact scaling; 0 when y < -126: the value would be subnormal)
+//   Z = sum_x e(x)   fp64, index order;   p(x) = fp32( (double) e(x) * (1 / Z) )   fp64 multiply, one rounding
+// logits: fp32 [rows][V];  probs out: fp32 [rows][V].
+// ---------------------------------------------------------------------------------
+int oracle_softmax_rows(const float* logits, long rows, int vocab, float* probs, int n_threads) {
+    if (rows < 0 || vocab <= 0) return -1;
+    static const float kLog2e = 1.44269504088896340736f;
+    // (ln 2)^k / k!, k = 0..7
+    static const float kC[8] = {1.0f, 6.93147180559945309e-1f, 2.40226506959100712e-1f, 5.55041086648215800e-2f,
+                                9.61812910762847716e-3f, 1.33335581464284434e-3f, 1.54035303933816099e-4f,
+                                1.52527338040598403e-5f};
+    parallel_for(rows, n_threads, [&](long r) {
+        const float* l = logits + r * static_cast<long>(vocab);
+        float* out = probs + r * static_cast<long>(vocab);
+        float m = l[0];
+        for (int x = 1; x < vocab; ++x) m = l[x] > m ? l[x] : m;
+        std::vector<float> e(vocab);
+        double Z = 0.0;
+        for (int x = 0; x < vocab; ++x) {
+            volatile float d = l[x] - m;
+            volatile float y = d * kLog2e;
+            float ex = 0.0f;
+            if (y >= -126.0f) {
+                const float n = std::nearbyintf(y);          // round to nearest even (default rounding mode)
+                volatile float f = y - n;
+                float g = kC[7];
+                for (int k = 6; k >= 0; --k) g = std::fmaf(g, f, kC[k]);
+                ex = std::ldexp(g, static_cast<int>(n));      // exact: g in [0.7, 1.5], n >= -126
+            }
+            e[x] = ex;
+            Z += static_cast<double>(ex);
+        }
+        const double inv = 1.0 / Z;
+        for (int x = 0; x < vocab; ++x) out[x] = static_cast<float>(static_cast<double>(e[x]) * inv);
+    });
+    return 0;
+}
+
+// ---------------------------------------------------------------------------------
 // Answer aggregation over the N branches of one question (Section 3.2 "majority voting";
 // Section 4.6 / Table "aggregation" for the confidence-weighted variants).
 //   mode 0 "vote": winner = answer with the largest count (weights == NULL) or the largest

@@ -23,7 +23,7 @@ EXPORTED_SYMBOLS = (
     "tts_attn_plan_drop",
     "tts_accept", "tts_majority_vote", "tts_confidence_max", "tts_greedy_search", "tts_grid_search", "tts_last_status",
     "tts_last_cuda_error", "tts_launch_count", "tts_strerror", "tts_verify_step_host",
-    "tts_profile_enable", "tts_profile_read", "tts_verify_attn_noalloc", "tts_kv_append", "tts_kv_rollback", "tts_accept_tree",
+    "tts_profile_enable", "tts_profile_read", "tts_debug_wait_timeout", "tts_verify_attn_noalloc", "tts_kv_append", "tts_kv_rollback", "tts_accept_tree",
 )
 
 
@@ -87,6 +87,7 @@ def load_library() -> ctypes.CDLL:
     lib.tts_last_cuda_error.argtypes = [vp]
     lib.tts_launch_count.argtypes = [vp]
     lib.tts_launch_count.restype = c_int64
+    lib.tts_debug_wait_timeout.argtypes = [vp, c_int64]
     lib.tts_profile_enable.argtypes = [vp, c_int]
     lib.tts_profile_read.argtypes = [vp, POINTER(c_float), POINTER(c_float), POINTER(c_int)]
     lib.tts_strerror.argtypes = [c_int]
@@ -215,6 +216,9 @@ class TtsContext:
         st = c_int(0)
         self._check(self._lib.tts_last_status(self._h, byref(st)), "tts_last_status")
         return st.value
+
+    def tts_debug_wait_timeout(self, limit_ns: int):
+        self._check(self._lib.tts_debug_wait_timeout(self._h, int(limit_ns)), "tts_debug_wait_timeout")
 
     def tts_profile_enable(self, on: bool):
         self._check(self._lib.tts_profile_enable(self._h, 1 if on else 0), "tts_profile_enable")

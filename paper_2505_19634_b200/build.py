@@ -15,7 +15,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libtts_b200.so"
-SOURCES = ["tts_api.cu", "attn_simt.cu", "attn_umma.cu", "attn_umma_t.cu", "attn_plan.cu", "attn_combine.cu", "accept.cu", "attn_noalloc.cu", "kv_cache.cu"]
+SOURCES = ["tts_api.cu", "attn_simt.cu", "attn_umma.cu", "attn_umma_t.cu", "attn_plan.cu", "attn_combine.cu", "accept.cu", "attn_noalloc.cu", "kv_cache.cu", "wait_probe.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr"]
 

@@ -486,6 +486,15 @@ int tts_last_status(tts_ctx* ctx, int* device_status) {
     return TTS_OK;
 }
 
+int tts_debug_wait_timeout(tts_ctx* ctx, int64_t limit_ns) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || limit_ns < 1000 || limit_ns > 1000ll * 1000 * 1000) return TTS_ERR_INVALID;
+    const cudaError_t e = launch_wait_probe(c->d_status, limit_ns, nullptr, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->launches += 1;
+    return TTS_OK;
+}
+
 int tts_profile_enable(tts_ctx* ctx, int on) {
     Ctx* c = reinterpret_cast<Ctx*>(ctx);
     if (!c) return TTS_ERR_INVALID;

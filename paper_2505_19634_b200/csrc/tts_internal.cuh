@@ -328,6 +328,7 @@ cudaError_t launch_kv_append(const void* k_new, const void* v_new, void* k_pages
                              const int32_t* branch_lens, int N, int R, int Hkv, int32_t* status, cudaStream_t st);
 cudaError_t launch_kv_rollback(int32_t* branch_lens, const int32_t* accepted_len, int N, int gamma, int32_t* status,
                                cudaStream_t st);
+cudaError_t launch_wait_probe(int32_t* status, long long limit_ns, int* gave_up, cudaStream_t st);
 int simt_rb_rows(int nr);
 constexpr int kSimtTileTokens = 64;
 

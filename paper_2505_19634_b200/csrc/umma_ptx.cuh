@@ -47,14 +47,14 @@ struct Abort {
 };
 
 // Bounded wait.  Returns false if the CTA is aborting (this or another wait ran out of time).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab, long long limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = global_ns();
     for (int spin = 0;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((spin & 63) == 63) {
             if (*ab.flag) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
+            if (global_ns() - t0 > limit_ns) {
                 *ab.flag = 1;
                 atomicMin(ab.status, (int)TTS_ERR_DEVICE_TIMEOUT);
                 return false;

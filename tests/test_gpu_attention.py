@@ -249,6 +249,24 @@ def test_debug_bounds_reports_bad_page_id_without_faulting():
     ctx.close()
 
 
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
+    """The give-up path of the bounded device-side waits: a probe kernel waits 1 ms for a signal nobody
+    sends; the status word then says timeout (-5), reading clears it, and attention calls on the same
+    context still give the right result."""
+    case = ti.make_attn_case(SMALL, 3)
+    want = oracle_out(case)
+    ctx = make_ctx(case, impl=tts.ATTN_TCGEN05_TOKEN_MAJOR, debug=True)
+    assert_attn_close(run_attn(case, ctx=ctx), want, what="before")
+    ctx.tts_debug_wait_timeout(1_000_000)
+    assert ctx.tts_last_status() == -5
+    assert ctx.tts_last_status() == 0
+    assert_attn_close(run_attn(case, ctx=ctx), want, what="after a timed-out wait")
+    for bad in (0, 999, 2_000_000_000):
+        with pytest.raises(tts.TtsError):
+            ctx.tts_debug_wait_timeout(bad)
+    ctx.close()
+
+
 @impl_param
 def test_debug_bounds_reports_a_block_index_past_the_table_row(impl):
     """branch_lens lives on the device, so the host cannot see a branch that claims more tokens than its

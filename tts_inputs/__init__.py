@@ -300,5 +300,40 @@ def make_accept_case(n_branches: int, gamma: int, vocab: int, sigma: float, seed
                       n_branches=n_branches, gamma=gamma, vocab=vocab)
 
 
+@dataclass
+class AcceptLogitsCase:
+    target_logits: np.ndarray  # [N][gamma+1][V] float32, or uint16 bf16 bits when made with bf16=True
+    draft_logits: np.ndarray   # [N][gamma][V]
+    draft_tokens: np.ndarray   # int32 [N][gamma]
+    uniforms: np.ndarray       # float32 [N][gamma+1]
+    n_branches: int
+    gamma: int
+    vocab: int
+    bf16: bool
+
+
+def make_accept_logits_case(n_branches: int, gamma: int, vocab: int, sigma: float, seed: int,
+                            draft_noise: Optional[float] = None, bf16: bool = False) -> AcceptLogitsCase:
+    """The logits behind `make_accept_case` (same recipe: N(0, sigma) logits, independent or target + noise),
+    kept as logits: fp32, or rounded to bf16 and carried as uint16 bit patterns.  Draft tokens are drawn from
+    the fp64 softmax of the (rounded) draft logits."""
+    rng = _rng(seed, 3)
+    tl = rng.standard_normal(size=(n_branches, gamma + 1, vocab), dtype=np.float32) * np.float32(sigma)
+    if draft_noise is None:
+        dl = rng.standard_normal(size=(n_branches, gamma, vocab), dtype=np.float32) * np.float32(sigma)
+    else:
+        dl = tl[:, :gamma, :] + rng.standard_normal(size=(n_branches, gamma, vocab),
+                                                    dtype=np.float32) * np.float32(draft_noise)
+    if bf16:
+        tl_out, dl_out = f32_to_bf16_bits(tl), f32_to_bf16_bits(dl)
+        dl = bf16_bits_to_f32(dl_out)
+    else:
+        tl_out, dl_out = tl, dl
+    toks = sample_from_rows(rng, _softmax_rows_f32(dl)) if gamma > 0 else np.zeros((n_branches, 0), np.int32)
+    u = uniforms24(rng, (n_branches, gamma + 1))
+    return AcceptLogitsCase(target_logits=tl_out, draft_logits=dl_out, draft_tokens=toks, uniforms=u,
+                            n_branches=n_branches, gamma=gamma, vocab=vocab, bf16=bf16)
+
+
 def with_branches(shape: AttnShape, **kw) -> AttnShape:
     return replace(shape, **kw)
