@@ -51,6 +51,7 @@ typedef enum {
 
 enum { TTS_MASK_CAUSAL = 0, TTS_MASK_TREE = 1 };
 enum { TTS_OUT_BF16 = 0, TTS_OUT_FP32 = 1 };
+enum { TTS_LOGITS_BF16 = 0, TTS_LOGITS_FP32 = 1 };
 /* Which attention kernel runs: AUTO picks tensor cores (tcgen05, TMEM accumulators) when the
  * stacked query rows per KV head make it worthwhile and CUDA cores otherwise.  TCGEN05 picks
  * between the two tensor-core kernels: TOKEN_MAJOR (KV tokens on the MMA M dimension, for at most
@@ -200,6 +201,28 @@ TTS_API int tts_accept(tts_ctx* ctx, const float* p_target, const float* q_draft
                int vocab, int32_t* accepted_len, int32_t* next_token);
 
 /*
+ * The same accept / resample rule fed with LOGITS (Section 2, "Speculative decoding": the rule compares
+ * the target's and the draft's token distributions; this entry point takes them before the softmax, so
+ * the fp32 probability tensors need not be materialised).  p_i = softmax(target_logits[b][i]) and q_i =
+ * softmax(draft_logits[b][i]) are formed inside the kernel, then everything is as in tts_accept.  The
+ * paper fixes no arithmetic for the softmax; the library's is stated step by step so that a host program
+ * can reproduce every decision bit for bit.  Per row l, with m = max_x l(x) and every step one correctly
+ * rounded operation:
+ *     d = l(x) - m (fp32);  y = d * log2(e) (fp32);  n = round-to-nearest-even(y);  f = y - n (exact);
+ *     g = sum_{k<8} (ln 2)^k / k! f^k by Horner's rule in fp32 fused multiply-adds, highest term first;
+ *     e(x) = g * 2^n (exact; 0 when y < -126);  Z = sum_x e(x) in fp64;  p(x) = fp32((double) e(x) * (1 / Z)).
+ * The fp64 sum is the only step whose result depends on the order of evaluation (relative 1e-16).  Callers
+ * apply a sampling temperature by scaling the logits beforehand.  Logits must be finite or -inf (a token
+ * that is ruled out), with at least one finite value per row.
+ *   target_logits device [n_branches][gamma+1][vocab], draft_logits device [n_branches][gamma][vocab],
+ *   both bf16 (TTS_LOGITS_BF16) or both fp32 (TTS_LOGITS_FP32), 16-byte aligned; the other arguments as
+ *   for tts_accept.  Only the rows up to the first rejection are read (twice: maximum, then sum).
+ */
+TTS_API int tts_accept_logits(tts_ctx* ctx, const void* target_logits, const void* draft_logits, int logits_dtype,
+                      const int32_t* draft_tokens, const float* uniforms, int n_branches, int gamma,
+                      int vocab, int32_t* accepted_len, int32_t* next_token);
+
+/*
  * Answer aggregation over the n branches of one question.  Host pointers, no GPU work.
  *   tts_majority_vote: winner = most frequent answer (weights == NULL, Section 3.2) or the answer
  *     with the largest weight sum ("vote" aggregation of Section 4.6); ties go to the answer whose
@@ -340,6 +363,18 @@ TTS_API int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host,
                          const void* const* v_pools, const int32_t* block_table_host,
                          int prefix_len, const int32_t* branch_lens_host, int n_branches, int gamma,
                          const float* p_target_host, const float* q_draft_host,
+                         const int32_t* draft_tokens_host, const float* uniforms_host, int vocab,
+                         void* out_host, int32_t* accepted_len_host, int32_t* next_token_host);
+
+/*
+ * tts_verify_step_host with the accept pass fed with logits (tts_accept_logits): target_logits_host
+ * [n_branches][gamma+1][vocab] and draft_logits_host [n_branches][gamma][vocab] in logits_dtype take the
+ * place of the two probability tensors (half the bytes over the host link when they are bf16).
+ */
+TTS_API int tts_verify_step_host_logits(tts_ctx* ctx, int n_layers, const void* q_host, const void* const* k_pools,
+                         const void* const* v_pools, const int32_t* block_table_host,
+                         int prefix_len, const int32_t* branch_lens_host, int n_branches, int gamma,
+                         const void* target_logits_host, const void* draft_logits_host, int logits_dtype,
                          const int32_t* draft_tokens_host, const float* uniforms_host, int vocab,
                          void* out_host, int32_t* accepted_len_host, int32_t* next_token_host);
 

@@ -16,12 +16,13 @@ _LIB_PATH = _PKG / "libtts_b200.so"
 
 MASK_CAUSAL, MASK_TREE = 0, 1
 OUT_BF16, OUT_FP32 = 0, 1
+LOGITS_BF16, LOGITS_FP32 = 0, 1
 ATTN_AUTO, ATTN_SIMT, ATTN_TCGEN05, ATTN_TCGEN05_TOKEN_MAJOR, ATTN_TCGEN05_ROW_MAJOR = 0, 1, 2, 3, 4
 
 EXPORTED_SYMBOLS = (
     "tts_create", "tts_destroy", "tts_set_stream", "tts_verify_attn", "tts_verify_attn_tree", "tts_attn_plan",
     "tts_attn_plan_drop",
-    "tts_accept", "tts_majority_vote", "tts_confidence_max", "tts_greedy_search", "tts_grid_search", "tts_last_status",
+    "tts_accept", "tts_accept_logits", "tts_verify_step_host_logits", "tts_majority_vote", "tts_confidence_max", "tts_greedy_search", "tts_grid_search", "tts_last_status",
     "tts_last_cuda_error", "tts_launch_count", "tts_strerror", "tts_verify_step_host",
     "tts_profile_enable", "tts_profile_read", "tts_debug_wait_timeout", "tts_verify_attn_noalloc", "tts_kv_append", "tts_kv_rollback", "tts_accept_tree",
 )
@@ -74,6 +75,9 @@ def load_library() -> ctypes.CDLL:
     lib.tts_attn_plan.argtypes = [vp, vp, c_int, vp, c_int, c_int]
     lib.tts_attn_plan_drop.argtypes = [vp]
     lib.tts_accept.argtypes = [vp, vp, vp, vp, vp, c_int, c_int, c_int, vp, vp]
+    lib.tts_accept_logits.argtypes = [vp, vp, vp, c_int, vp, vp, c_int, c_int, c_int, vp, vp]
+    lib.tts_verify_step_host_logits.argtypes = [vp, c_int, vp, POINTER(c_void_p), POINTER(c_void_p), vp, c_int, vp,
+                                                c_int, c_int, vp, vp, c_int, vp, vp, c_int, vp, vp, vp]
     lib.tts_accept_tree.argtypes = [vp, vp, vp, vp, vp, vp, c_int, c_int, c_int, vp, vp, vp]
     lib.tts_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, c_int, vp, c_int, c_int]
     lib.tts_kv_rollback.argtypes = [vp, vp, vp, c_int, c_int]
@@ -195,6 +199,12 @@ class TtsContext:
                                          int(n_branches), int(gamma), int(vocab), _ptr(accepted_len),
                                          _ptr(next_token)), "tts_accept")
 
+    def tts_accept_logits(self, target_logits, draft_logits, logits_dtype: int, draft_tokens, uniforms,
+                          n_branches: int, gamma: int, vocab: int, accepted_len, next_token):
+        self._check(self._lib.tts_accept_logits(self._h, _ptr(target_logits), _ptr(draft_logits), int(logits_dtype),
+                                                _ptr(draft_tokens), _ptr(uniforms), int(n_branches), int(gamma),
+                                                int(vocab), _ptr(accepted_len), _ptr(next_token)), "tts_accept_logits")
+
     def tts_accept_tree(self, p_target, q_draft, draft_tokens, tree_parents, uniforms, n_branches: int, n_nodes: int,
                         vocab: int, accepted_len, last_node, next_token):
         self._check(self._lib.tts_accept_tree(self._h, _ptr(p_target), _ptr(q_draft), _ptr(draft_tokens),
@@ -243,6 +253,22 @@ class TtsContext:
             _ptr(branch_lens_host), int(n_branches), int(gamma), _ptr(p_target_host), _ptr(q_draft_host),
             _ptr(draft_tokens_host), _ptr(uniforms_host), int(vocab), _ptr(out_host), _ptr(accepted_len_host),
             _ptr(next_token_host)), "tts_verify_step_host")
+
+
+def _step_host_logits(self, n_layers: int, q_host, k_pools: Sequence, v_pools: Sequence, block_table_host,
+                      prefix_len: int, branch_lens_host, n_branches: int, gamma: int, target_logits_host,
+                      draft_logits_host, logits_dtype: int, draft_tokens_host, uniforms_host, vocab: int, out_host,
+                      accepted_len_host, next_token_host):
+    ka = (c_void_p * n_layers)(*[_ptr(k).value for k in k_pools])
+    va = (c_void_p * n_layers)(*[_ptr(v).value for v in v_pools])
+    self._check(self._lib.tts_verify_step_host_logits(
+        self._h, int(n_layers), _ptr(q_host), ka, va, _ptr(block_table_host), int(prefix_len),
+        _ptr(branch_lens_host), int(n_branches), int(gamma), _ptr(target_logits_host), _ptr(draft_logits_host),
+        int(logits_dtype), _ptr(draft_tokens_host), _ptr(uniforms_host), int(vocab), _ptr(out_host),
+        _ptr(accepted_len_host), _ptr(next_token_host)), "tts_verify_step_host_logits")
+
+
+TtsContext.tts_verify_step_host_logits = _step_host_logits
 
 
 def tts_verify_attn_noalloc(q, k_pages, v_pages, block_table, max_blocks_per_branch: int, prefix_len: int,

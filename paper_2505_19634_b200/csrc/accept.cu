@@ -39,9 +39,78 @@ __device__ __forceinline__ float weight(float p, float q, bool residual) {
     return d > 0.f ? d : 0.f;
 }
 
+// Where the weights of the final draw come from: four consecutive tokens at a time.  `Raw` is what one
+// thread loads for them (all loads of a batch are issued before the first is used); weights() turns it into
+// the four fp32 weights, max(0, p - q) for a residual draw and p otherwise.
+struct ProbRows {                                   // rows of probabilities
+    const float* pk; const float* qk;
+    struct Raw { float4 p, q; };
+    __device__ __forceinline__ Raw load(int x0, bool residual) const {
+        Raw r;
+        r.p = __ldg(reinterpret_cast<const float4*>(pk + x0));
+        r.q = residual ? __ldg(reinterpret_cast<const float4*>(qk + x0)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        return r;
+    }
+    __device__ __forceinline__ void weights(const Raw& r, bool residual, float* w) const {
+        w[0] = weight(r.p.x, r.q.x, residual); w[1] = weight(r.p.y, r.q.y, residual);
+        w[2] = weight(r.p.z, r.q.z, residual); w[3] = weight(r.p.w, r.q.w, residual);
+    }
+};
+
+// Probabilities from logits, every step one correctly rounded operation so that a host program can
+// reproduce them bit for bit: d = l - max (fp32), y = d * log2(e) (fp32), n = round-to-nearest-even(y),
+// f = y - n (exact), g = eight-term Taylor polynomial of 2^f by fp32 fused multiply-adds, e = g * 2^n (exact;
+// 0 when y < -126), p = fp32((double) e * (1 / Z)) with Z the fp64 sum of the row's e.
+__device__ __forceinline__ float exp_rel(float l, float m) {
+    const float y = __fmul_rn(__fsub_rn(l, m), 1.44269504088896340736f);
+    if (!(y >= -126.f)) return 0.f;
+    const float n = rintf(y);
+    const float f = __fsub_rn(y, n);
+    float g = 1.52527338040598403e-5f;                                  // (ln 2)^k / k!, k = 7 .. 0
+    g = __fmaf_rn(g, f, 1.54035303933816099e-4f);
+    g = __fmaf_rn(g, f, 1.33335581464284434e-3f);
+    g = __fmaf_rn(g, f, 9.61812910762847716e-3f);
+    g = __fmaf_rn(g, f, 5.55041086648215800e-2f);
+    g = __fmaf_rn(g, f, 2.40226506959100712e-1f);
+    g = __fmaf_rn(g, f, 6.93147180559945309e-1f);
+    g = __fmaf_rn(g, f, 1.0f);
+    return __fmul_rn(g, __int_as_float(((int)n + 127) << 23));
+}
+__device__ __forceinline__ float prob_of(float l, float m, double inv_z) {
+    return __double2float_rn(__dmul_rn((double)exp_rel(l, m), inv_z));
+}
+
+__device__ __forceinline__ float4 load4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
+    const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
+    return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u),
+                       __uint_as_float(v.y << 16), __uint_as_float(v.y & 0xffff0000u));
+}
+
+template <typename T>
+struct LogitRows {                                  // rows of logits with their maxima and 1 / normalisers
+    const T* lp; const T* lq;
+    float mp, mq;
+    double inv_p, inv_q;
+    struct Raw { float4 p, q; };
+    __device__ __forceinline__ Raw load(int x0, bool residual) const {
+        Raw r;
+        r.p = load4(lp + x0);
+        r.q = residual ? load4(lq + x0) : make_float4(0.f, 0.f, 0.f, 0.f);
+        return r;
+    }
+    __device__ __forceinline__ void weights(const Raw& r, bool residual, float* w) const {
+        const float lpv[4] = {r.p.x, r.p.y, r.p.z, r.p.w}, lqv[4] = {r.q.x, r.q.y, r.q.z, r.q.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            w[e] = weight(prob_of(lpv[e], mp, inv_p), residual ? prob_of(lqv[e], mq, inv_q) : 0.f, residual);
+    }
+};
+
 // Steps 2 and 3 for one branch, by the whole CTA: the draw with u_final from norm(max(0, p - q)) (residual;
 // from p if that is identically zero) or from p.  tile_sum, s_last_pos (-1) and s_redo (0) are shared scratch.
-__device__ __forceinline__ void draw_token(const float* __restrict__ pk, const float* __restrict__ qk, bool residual,
+template <class Rows>
+__device__ __forceinline__ void draw_token(const Rows& rows, bool residual,
                                            float u_final, int vocab, double* tile_sum, int* s_last_pos_p, int* s_redo_p,
                                            int32_t* next_token_out) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -57,15 +126,11 @@ __device__ __forceinline__ void draw_token(const float* __restrict__ pk, const f
         // to keep many loads in flight to pull its share of the bandwidth)
         constexpr int kSweepBatch = 4, kWarps = kAccThreads / 32;
         for (int j0 = warp; j0 < n_tiles; j0 += kWarps * kSweepBatch) {
-            float4 pv[kSweepBatch], qv[kSweepBatch];
+            typename Rows::Raw raw[kSweepBatch];
 #pragma unroll
             for (int k = 0; k < kSweepBatch; ++k) {
                 const int x0 = (j0 + k * kWarps) * kTileElems + lane * 4;
-                pv[k] = qv[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (j0 + k * kWarps < n_tiles && x0 < vocab) {      // vocab % 4 == 0: whole float4 in range
-                    pv[k] = __ldg(reinterpret_cast<const float4*>(pk + x0));
-                    if (residual) qv[k] = __ldg(reinterpret_cast<const float4*>(qk + x0));
-                }
+                if (j0 + k * kWarps < n_tiles && x0 < vocab) raw[k] = rows.load(x0, residual);   // vocab % 4 == 0: four tokens in range
             }
 #pragma unroll
             for (int k = 0; k < kSweepBatch; ++k) {
@@ -74,8 +139,9 @@ __device__ __forceinline__ void draw_token(const float* __restrict__ pk, const f
                 const int x0 = j * kTileElems + lane * 4;
                 double s = 0.0;
                 if (x0 < vocab) {
-                    const float w0 = weight(pv[k].x, qv[k].x, residual), w1 = weight(pv[k].y, qv[k].y, residual);
-                    const float w2 = weight(pv[k].z, qv[k].z, residual), w3 = weight(pv[k].w, qv[k].w, residual);
+                    float w[4];
+                    rows.weights(raw[k], residual, w);
+                    const float w0 = w[0], w1 = w[1], w2 = w[2], w3 = w[3];
                     s = (double)w0 + (double)w1 + (double)w2 + (double)w3;
                     if (w3 > 0.f) last_pos = max(last_pos, x0 + 3); else if (w2 > 0.f) last_pos = max(last_pos, x0 + 2);
                     else if (w1 > 0.f) last_pos = max(last_pos, x0 + 1); else if (w0 > 0.f) last_pos = max(last_pos, x0);
@@ -137,13 +203,7 @@ __device__ __forceinline__ void draw_token(const float* __restrict__ pk, const f
             if (tile >= 0) {
                 const int x0 = tile * kTileElems + lane * 4;
                 float w[4] = {0.f, 0.f, 0.f, 0.f};
-                if (x0 < vocab) {
-                    const float4 pv = *reinterpret_cast<const float4*>(pk + x0);
-                    float4 qv = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (residual) qv = *reinterpret_cast<const float4*>(qk + x0);
-                    w[0] = weight(pv.x, qv.x, residual); w[1] = weight(pv.y, qv.y, residual);
-                    w[2] = weight(pv.z, qv.z, residual); w[3] = weight(pv.w, qv.w, residual);
-                }
+                if (x0 < vocab) rows.weights(rows.load(x0, residual), residual, w);
                 const double ls = (double)w[0] + (double)w[1] + (double)w[2] + (double)w[3];
                 const double lincl = warp_incl_scan(ls, lane);
                 const unsigned lhit = __ballot_sync(0xffffffffu, base + lincl > t);
@@ -207,7 +267,99 @@ accept_kernel(const float* __restrict__ p_target, const float* __restrict__ q_dr
     const int k = s_k;
     const float* pk = P + (size_t)k * vocab;
     const float* qk = Q + (size_t)(k < gamma ? k : 0) * vocab;
-    draw_token(pk, qk, k < gamma, U[gamma], vocab, tile_sum, &s_last_pos, &s_redo, next_token + b);
+    draw_token(ProbRows{pk, qk}, k < gamma, U[gamma], vocab, tile_sum, &s_last_pos, &s_redo, next_token + b);
+}
+
+// Maximum and normaliser of one or two rows of logits, by the whole CTA: one pass for the maxima, one for the
+// sums of exp_rel (fp64).  red is shared scratch of 64 doubles.  All threads return the same values.
+template <typename T>
+__device__ void rows_max_and_norm(const T* row_a, const T* row_b, int vocab, double* red, float* m_out, double* inv_out) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int kWarps = kAccThreads / 32;
+    const int n_rows = row_b ? 2 : 1;
+    float m[2] = {-INFINITY, -INFINITY};
+    for (int x0 = tid * 4; x0 < vocab; x0 += kAccThreads * 4) {
+        const float4 a = load4(row_a + x0);
+        m[0] = fmaxf(m[0], fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)));
+        if (row_b) {
+            const float4 c = load4(row_b + x0);
+            m[1] = fmaxf(m[1], fmaxf(fmaxf(c.x, c.y), fmaxf(c.z, c.w)));
+        }
+    }
+    float* redf = reinterpret_cast<float*>(red);
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m[r] = fmaxf(m[r], __shfl_xor_sync(0xffffffffu, m[r], o));
+        if (lane == 0) redf[r * kWarps + warp] = m[r];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        float v = redf[r * kWarps + lane];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+        m[r] = v;
+    }
+    __syncthreads();
+    double z[2] = {0.0, 0.0};
+    for (int x0 = tid * 4; x0 < vocab; x0 += kAccThreads * 4) {
+        const float4 a = load4(row_a + x0);
+        z[0] += ((double)exp_rel(a.x, m[0]) + (double)exp_rel(a.y, m[0])) + ((double)exp_rel(a.z, m[0]) + (double)exp_rel(a.w, m[0]));
+        if (row_b) {
+            const float4 c = load4(row_b + x0);
+            z[1] += ((double)exp_rel(c.x, m[1]) + (double)exp_rel(c.y, m[1])) + ((double)exp_rel(c.z, m[1]) + (double)exp_rel(c.w, m[1]));
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        z[r] = warp_sum(z[r]);
+        if (lane == 0) red[r * kWarps + warp] = z[r];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < 2; ++r) z[r] = warp_sum(red[r * kWarps + lane]);
+    __syncthreads();
+    for (int r = 0; r < n_rows; ++r) { m_out[r] = m[r]; inv_out[r] = 1.0 / z[r]; }
+}
+
+// The accept rule fed with logits: the probabilities the tests and the final draw need are formed on the way
+// (prob_of), position by position, so only the rows up to the first rejection are read.
+template <typename T>
+__global__ void __launch_bounds__(kAccThreads)
+accept_logits_kernel(const T* __restrict__ target_logits, const T* __restrict__ draft_logits,
+                     const int32_t* __restrict__ draft_tokens, const float* __restrict__ uniforms, int gamma,
+                     int vocab, int32_t* __restrict__ accepted_len, int32_t* __restrict__ next_token,
+                     int32_t* status) {
+    __shared__ double tile_sum[kMaxTiles];
+    __shared__ double red[64];
+    __shared__ int s_last_pos, s_redo;
+    static_assert(kAccThreads == 1024, "the block reductions assume 32 warps");
+
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const T* P = target_logits + (size_t)b * (gamma + 1) * vocab;
+    const T* Q = draft_logits + (size_t)b * gamma * vocab;
+    const float* U = uniforms + (size_t)b * (gamma + 1);
+
+    int k = gamma;
+    float m[2] = {0.f, 0.f};
+    double inv[2] = {1.0, 1.0};
+    for (int i = 0; i < gamma; ++i) {
+        const T* pi = P + (size_t)i * vocab;
+        const T* qi = Q + (size_t)i * vocab;
+        rows_max_and_norm(pi, qi, vocab, red, m, inv);
+        int x = draft_tokens[(size_t)b * gamma + i];                     // the same for all threads
+        if (x < 0 || x >= vocab) { if (tid == 0) atomicMin(status, (int)TTS_ERR_DEVICE_BOUNDS); x = 0; }
+        const float p = prob_of((float)pi[x], m[0], inv[0]);
+        const float q = prob_of((float)qi[x], m[1], inv[1]);
+        const float uq = __fmul_rn(U[i], q);
+        if (!(p > 0.f && uq <= p)) { k = i; break; }                     // uniform over the block
+    }
+    if (k == gamma) rows_max_and_norm<T>(P + (size_t)gamma * vocab, nullptr, vocab, red, m, inv);
+    if (tid == 0) { accepted_len[b] = k; s_last_pos = -1; s_redo = 0; }
+    __syncthreads();
+    const LogitRows<T> rows{P + (size_t)k * vocab, Q + (size_t)(k < gamma ? k : 0) * vocab, m[0], m[1], inv[0], inv[1]};
+    draw_token(rows, k < gamma, U[gamma], vocab, tile_sum, &s_last_pos, &s_redo, next_token + b);
 }
 
 // The same for a draft tree (n nodes per branch, at most kMaxTreeRows): node i passes iff
@@ -271,7 +423,7 @@ accept_tree_kernel(const float* __restrict__ p_target, const float* __restrict__
     __syncthreads();
     const float* pk = P + (size_t)s_row * vocab;
     const float* qk = Q + (size_t)(s_qrow >= 0 ? s_qrow : 0) * vocab;
-    draw_token(pk, qk, s_qrow >= 0, U[n], vocab, tile_sum, &s_last_pos, &s_redo, next_token + b);
+    draw_token(ProbRows{pk, qk}, s_qrow >= 0, U[n], vocab, tile_sum, &s_last_pos, &s_redo, next_token + b);
 }
 
 }  // namespace
@@ -282,6 +434,20 @@ cudaError_t launch_accept(const float* p_target, const float* q_draft, const int
                           cudaStream_t st) {
     accept_kernel<<<n_branches, kAccThreads, 0, st>>>(p_target, q_draft, draft_tokens, uniforms,
                                                       gamma, vocab, accepted_len, next_token, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_accept_logits(const void* target_logits, const void* draft_logits, int logits_dtype,
+                                 const int32_t* draft_tokens, const float* uniforms, int n_branches, int gamma, int vocab,
+                                 int32_t* accepted_len, int32_t* next_token, int32_t* status, cudaStream_t st) {
+    if (logits_dtype == TTS_LOGITS_BF16)
+        accept_logits_kernel<__nv_bfloat16><<<n_branches, kAccThreads, 0, st>>>(
+            static_cast<const __nv_bfloat16*>(target_logits), static_cast<const __nv_bfloat16*>(draft_logits), draft_tokens,
+            uniforms, gamma, vocab, accepted_len, next_token, status);
+    else
+        accept_logits_kernel<float><<<n_branches, kAccThreads, 0, st>>>(
+            static_cast<const float*>(target_logits), static_cast<const float*>(draft_logits), draft_tokens, uniforms, gamma,
+            vocab, accepted_len, next_token, status);
     return cudaGetLastError();
 }
 

@@ -325,6 +325,23 @@ int tts_accept(tts_ctx* ctx, const float* p_target, const float* q_draft, const 
     return TTS_OK;
 }
 
+int tts_accept_logits(tts_ctx* ctx, const void* target_logits, const void* draft_logits, int logits_dtype,
+                      const int32_t* draft_tokens, const float* uniforms, int n_branches, int gamma, int vocab,
+                      int32_t* accepted_len, int32_t* next_token) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !target_logits || !uniforms || !accepted_len || !next_token) return TTS_ERR_INVALID;
+    if (logits_dtype != TTS_LOGITS_BF16 && logits_dtype != TTS_LOGITS_FP32) return TTS_ERR_UNSUPPORTED;
+    if (gamma < 0 || n_branches < 1) return TTS_ERR_INVALID;
+    if (gamma > 0 && (!draft_logits || !draft_tokens)) return TTS_ERR_INVALID;
+    if (vocab < 4 || vocab % 4 != 0 || vocab > 524288) return TTS_ERR_INVALID;
+    if (!aligned16(target_logits) || (draft_logits && !aligned16(draft_logits))) return TTS_ERR_INVALID;
+    cudaError_t e = launch_accept_logits(target_logits, draft_logits, logits_dtype, draft_tokens, uniforms, n_branches,
+                                         gamma, vocab, accepted_len, next_token, c->d_status, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->launches += 1;
+    return TTS_OK;
+}
+
 int tts_accept_tree(tts_ctx* ctx, const float* p_target, const float* q_draft, const int32_t* draft_tokens,
                     const int32_t* tree_parents, const float* uniforms, int n_branches, int n_nodes, int vocab,
                     int32_t* accepted_len, int32_t* last_node, int32_t* next_token) {
@@ -552,12 +569,19 @@ const char* tts_strerror(int status) {
     }
 }
 
-int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const void* const* k_pools,
-                         const void* const* v_pools, const int32_t* block_table_host, int prefix_len,
-                         const int32_t* branch_lens_host, int n_branches, int gamma,
-                         const float* p_target_host, const float* q_draft_host,
-                         const int32_t* draft_tokens_host, const float* uniforms_host, int vocab,
-                         void* out_host, int32_t* accepted_len_host, int32_t* next_token_host) {
+}  // extern "C"
+
+namespace {
+
+// The end-to-end step from host buffers.  dist_elt: bytes per element of the two distribution tensors (4: fp32
+// probabilities or logits, 2: bf16 logits); logits_dtype < 0: they are probabilities.
+int step_host(tts_ctx* ctx, int n_layers, const void* q_host, const void* const* k_pools,
+              const void* const* v_pools, const int32_t* block_table_host, int prefix_len,
+              const int32_t* branch_lens_host, int n_branches, int gamma,
+              const void* p_target_host, const void* q_draft_host, int logits_dtype,
+              const int32_t* draft_tokens_host, const float* uniforms_host, int vocab,
+              void* out_host, int32_t* accepted_len_host, int32_t* next_token_host) {
+    const size_t dist_elt = logits_dtype == TTS_LOGITS_BF16 ? 2 : 4;
     Ctx* c = reinterpret_cast<Ctx*>(ctx);
     if (!c || n_layers < 1 || !q_host || !k_pools || !v_pools || !block_table_host || !branch_lens_host ||
         !p_target_host || !uniforms_host || !out_host || !accepted_len_host || !next_token_host)
@@ -572,8 +596,8 @@ int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const v
     const size_t o_layer = (size_t)n_branches * (gamma + 1) * f.n_q_heads * kHeadDim * out_elt;
     auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
     const size_t bt_b = up((size_t)n_branches * f.max_blocks_per_branch * 4), bl_b = up((size_t)n_branches * 4);
-    const size_t pt_b = up((size_t)n_branches * (gamma + 1) * vocab * 4);
-    const size_t qd_b = up((size_t)n_branches * gamma * vocab * 4);
+    const size_t pt_b = up((size_t)n_branches * (gamma + 1) * vocab * dist_elt);
+    const size_t qd_b = up((size_t)n_branches * gamma * vocab * dist_elt);
     const size_t dt_b = up((size_t)n_branches * gamma * 4), un_b = up((size_t)n_branches * (gamma + 1) * 4);
     const size_t res_b = up((size_t)n_branches * 4);
     const size_t need = up(q_layer) * n_layers + up(o_layer) * n_layers + bt_b + bl_b + pt_b + qd_b + dt_b +
@@ -589,8 +613,8 @@ int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const v
     char* d_o = base;               base += up(o_layer) * n_layers;
     int32_t* d_bt = (int32_t*)base; base += bt_b;
     int32_t* d_bl = (int32_t*)base; base += bl_b;
-    float* d_pt = (float*)base;     base += pt_b;
-    float* d_qd = (float*)base;     base += qd_b;
+    char* d_pt = base;              base += pt_b;
+    char* d_qd = base;              base += qd_b;
     int32_t* d_dt = (int32_t*)base; base += dt_b;
     float* d_un = (float*)base;     base += un_b;
     int32_t* d_al = (int32_t*)base; base += res_b;
@@ -651,9 +675,9 @@ int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const v
         TTS_CK(copy_q(l0, l1, up_st));
         TTS_CK(cudaEventRecord(ev_q[ch], up_st));
     }
-    TTS_CK(cudaMemcpyAsync(d_pt, p_target_host, (size_t)n_branches * (gamma + 1) * vocab * 4, cudaMemcpyHostToDevice, up_st));
+    TTS_CK(cudaMemcpyAsync(d_pt, p_target_host, (size_t)n_branches * (gamma + 1) * vocab * dist_elt, cudaMemcpyHostToDevice, up_st));
     if (gamma > 0) {
-        TTS_CK(cudaMemcpyAsync(d_qd, q_draft_host, (size_t)n_branches * gamma * vocab * 4, cudaMemcpyHostToDevice, up_st));
+        TTS_CK(cudaMemcpyAsync(d_qd, q_draft_host, (size_t)n_branches * gamma * vocab * dist_elt, cudaMemcpyHostToDevice, up_st));
         TTS_CK(cudaMemcpyAsync(d_dt, draft_tokens_host, (size_t)n_branches * gamma * 4, cudaMemcpyHostToDevice, up_st));
     }
     TTS_CK(cudaMemcpyAsync(d_un, uniforms_host, (size_t)n_branches * (gamma + 1) * 4, cudaMemcpyHostToDevice, up_st));
@@ -677,8 +701,11 @@ int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const v
         TTS_CK(copy_o(l0, l1, down_st));
     }
     TTS_CK(cudaStreamWaitEvent(st, ev_acc, 0));
-    int rc = tts_accept(ctx, d_pt, gamma > 0 ? d_qd : nullptr, gamma > 0 ? d_dt : nullptr, d_un, n_branches, gamma,
-                        vocab, d_al, d_nt);
+    int rc = logits_dtype < 0
+                 ? tts_accept(ctx, (const float*)d_pt, gamma > 0 ? (const float*)d_qd : nullptr, gamma > 0 ? d_dt : nullptr, d_un,
+                              n_branches, gamma, vocab, d_al, d_nt)
+                 : tts_accept_logits(ctx, d_pt, gamma > 0 ? d_qd : nullptr, logits_dtype, gamma > 0 ? d_dt : nullptr, d_un,
+                                     n_branches, gamma, vocab, d_al, d_nt);
     if (rc != TTS_OK) { drain(); return rc; }
     TTS_CK(cudaMemcpyAsync(accepted_len_host, d_al, (size_t)n_branches * 4, cudaMemcpyDeviceToHost, st));
     TTS_CK(cudaMemcpyAsync(next_token_host, d_nt, (size_t)n_branches * 4, cudaMemcpyDeviceToHost, st));
@@ -688,6 +715,33 @@ int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const v
     TTS_CK(cudaStreamSynchronize(up_st));
 #undef TTS_CK
     return TTS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const void* const* k_pools,
+                         const void* const* v_pools, const int32_t* block_table_host, int prefix_len,
+                         const int32_t* branch_lens_host, int n_branches, int gamma,
+                         const float* p_target_host, const float* q_draft_host,
+                         const int32_t* draft_tokens_host, const float* uniforms_host, int vocab,
+                         void* out_host, int32_t* accepted_len_host, int32_t* next_token_host) {
+    return step_host(ctx, n_layers, q_host, k_pools, v_pools, block_table_host, prefix_len, branch_lens_host, n_branches,
+                     gamma, p_target_host, q_draft_host, -1, draft_tokens_host, uniforms_host, vocab, out_host,
+                     accepted_len_host, next_token_host);
+}
+
+int tts_verify_step_host_logits(tts_ctx* ctx, int n_layers, const void* q_host, const void* const* k_pools,
+                                const void* const* v_pools, const int32_t* block_table_host, int prefix_len,
+                                const int32_t* branch_lens_host, int n_branches, int gamma,
+                                const void* target_logits_host, const void* draft_logits_host, int logits_dtype,
+                                const int32_t* draft_tokens_host, const float* uniforms_host, int vocab,
+                                void* out_host, int32_t* accepted_len_host, int32_t* next_token_host) {
+    if (logits_dtype != TTS_LOGITS_BF16 && logits_dtype != TTS_LOGITS_FP32) return TTS_ERR_UNSUPPORTED;
+    return step_host(ctx, n_layers, q_host, k_pools, v_pools, block_table_host, prefix_len, branch_lens_host, n_branches,
+                     gamma, target_logits_host, draft_logits_host, logits_dtype, draft_tokens_host, uniforms_host, vocab,
+                     out_host, accepted_len_host, next_token_host);
 }
 
 }  // extern "C"

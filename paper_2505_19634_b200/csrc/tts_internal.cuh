@@ -319,6 +319,9 @@ cudaError_t launch_accept(const float* p_target, const float* q_draft, const int
                           const float* uniforms, int n_branches, int gamma, int vocab,
                           int32_t* accepted_len, int32_t* next_token, int32_t* status,
                           cudaStream_t st);
+cudaError_t launch_accept_logits(const void* target_logits, const void* draft_logits, int logits_dtype,
+                                 const int32_t* draft_tokens, const float* uniforms, int n_branches, int gamma, int vocab,
+                                 int32_t* accepted_len, int32_t* next_token, int32_t* status, cudaStream_t st);
 cudaError_t launch_accept_tree(const float* p_target, const float* q_draft, const int32_t* draft_tokens,
                                const int32_t* tree_parents, const float* uniforms, int n_branches, int n_nodes, int vocab,
                                int32_t* accepted_len, int32_t* last_node, int32_t* next_token, int32_t* status,
