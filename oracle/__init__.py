@@ -101,6 +101,29 @@ def verify_attn(q, k_pages, v_pages, block_table, prefix_len, branch_lens, gamma
     return out
 
 
+def verify_attn_groups(q, k_pages, v_pages, block_table, group_sizes, group_prefix_lens, branch_lens, gamma,
+                       n_threads=None):
+    """Several questions in one call (the multi-request setting of the paper's appendix: #Req questions, each
+    with B branches that share that question's prompt).  Branches are numbered group by group; the branches
+    of group g share a prefix of group_prefix_lens[g] tokens, listed first in their block-table rows.  By
+    definition the groups do not interact: the result for a branch is the single-question result
+    (`verify_attn`) for its group alone, with that group's prefix length.  Returns fp64 out [N][R][Hq][D]."""
+    q = np.ascontiguousarray(q, dtype=np.uint16)
+    block_table = np.ascontiguousarray(block_table, dtype=np.int32)
+    branch_lens = np.ascontiguousarray(branch_lens, dtype=np.int32)
+    sizes = [int(v) for v in group_sizes]
+    assert sum(sizes) == q.shape[0] and len(sizes) == len(group_prefix_lens)
+    out = np.zeros(q.shape, dtype=np.float64)
+    b0 = 0
+    for size, prefix_len in zip(sizes, group_prefix_lens):
+        b1 = b0 + size
+        if size > 0:
+            out[b0:b1] = verify_attn(q[b0:b1], k_pages, v_pages, block_table[b0:b1], int(prefix_len),
+                                     branch_lens[b0:b1], gamma, n_threads=n_threads)
+        b0 = b1
+    return out
+
+
 def accept(p_target, q_draft, draft_tokens, uniforms, n_threads=None):
     """Speculative-sampling accept/resample.  Returns (accepted_len, next_token, near_flags)."""
     p_target = np.ascontiguousarray(p_target, dtype=np.float32)

@@ -207,3 +207,57 @@ def test_kv_byte_accounting_matches_the_paper():
     assert ti.CONFIGS["tiny"].unique_kv_bytes() == 1310720
     assert ti.CONFIGS["3b"].unique_kv_bytes() == 17301504
     assert ti.CONFIGS["32b"].unique_kv_bytes() == 270532608
+
+
+# ---- several prefix groups per call (multi-request setting of the paper's appendix) ----
+def _group_case(seed=4, **kw):
+    args = dict(n_q_heads=4, n_kv_heads=2, gamma=2, group_sizes=(2, 1, 3), group_prefix_lens=(32, 0, 48),
+                branch_lens=(19, 3, 40, 7, 33, 16), seed=seed, extra_pages=3)
+    args.update(kw)
+    return ti.make_group_case(**args)
+
+
+def _run_groups(c):
+    return oracle.verify_attn_groups(c.q, c.k_pages, c.v_pages, c.block_table, c.group_sizes, c.group_prefix_lens,
+                                     c.branch_lens, c.gamma)
+
+
+def test_groups_match_dense_brute_force_per_branch():
+    """Every branch against the dense reference run on that branch alone with ITS group's prefix length
+    (explicit mask matrix, dense softmax: code that knows nothing about groups)."""
+    c = _group_case()
+    ti.poison_unused_slots_groups(c)
+    got = _run_groups(c)
+    assert np.isfinite(got).all()
+    group = c.group_of_branch()
+    for b in range(c.n_branches):
+        one = ti.AttnCase(shape=ti.AttnShape("one", n_q_heads=4, n_kv_heads=2, prefix_len=int(c.group_prefix_lens[group[b]]),
+                                             n_branches=1, gamma=2, branch_lens=(int(c.branch_lens[b]),)),
+                          q=c.q[b:b + 1], k_pages=c.k_pages, v_pages=c.v_pages, block_table=c.block_table[b:b + 1],
+                          branch_lens=c.branch_lens[b:b + 1], prefix_len=int(c.group_prefix_lens[group[b]]),
+                          num_pages=c.num_pages, max_blocks=c.max_blocks)
+        np.testing.assert_allclose(got[b:b + 1], dense_reference(one), rtol=1e-11, atol=1e-13)
+
+
+def test_one_group_is_the_single_question_call_bit_for_bit():
+    case = ti.make_attn_case(small_shape(), 6)
+    want = run(case)
+    got = oracle.verify_attn_groups(case.q, case.k_pages, case.v_pages, case.block_table, [3], [case.prefix_len],
+                                    case.branch_lens, case.shape.gamma)
+    assert np.array_equal(got, want)
+
+
+def test_groups_do_not_interact():
+    """Overwriting the prefix keys and values of group 0 changes the rows of group 0 and leaves every other
+    group's rows bit-identical; the block table really shares the prefix pages inside a group only."""
+    c = _group_case()
+    base = _run_groups(c)
+    n_pre0 = int(c.group_prefix_lens[0]) // 16
+    shared = c.block_table[0, :n_pre0]
+    assert np.array_equal(c.block_table[1, :n_pre0], shared)                       # shared inside group 0
+    assert not np.isin(c.block_table[2:], shared).any()                            # and nowhere else
+    c.k_pages[shared] = ti.f32_to_bf16_bits(np.full(c.k_pages[shared].shape, 0.5, np.float32))
+    c.v_pages[shared] = ti.f32_to_bf16_bits(np.full(c.v_pages[shared].shape, -2.0, np.float32))
+    moved = _run_groups(c)
+    assert np.array_equal(moved[2:], base[2:])
+    assert np.abs(moved[:2] - base[:2]).max() > 1e-3

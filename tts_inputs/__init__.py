@@ -218,6 +218,96 @@ def poison_unused_slots(case: AttnCase, bits: int = 0x7FC0) -> None:
 
 
 # --------------------------------------------------------------------------- #
+# several prefix groups per call (several questions in flight, each with its own shared prompt)
+# --------------------------------------------------------------------------- #
+@dataclass
+class GroupCase:
+    """Branches numbered group by group; the branches of group g share the first group_prefix_lens[g] / 16
+    entries of their block-table rows."""
+    n_q_heads: int
+    n_kv_heads: int
+    gamma: int
+    group_sizes: np.ndarray        # int32 [n_groups]
+    group_prefix_lens: np.ndarray  # int32 [n_groups], multiples of PAGE
+    q: np.ndarray
+    k_pages: np.ndarray
+    v_pages: np.ndarray
+    block_table: np.ndarray        # int32 [N][max_blocks]
+    branch_lens: np.ndarray        # int32 [N]
+    num_pages: int
+    max_blocks: int
+
+    @property
+    def n_branches(self) -> int:
+        return int(self.group_sizes.sum())
+
+    def group_of_branch(self) -> np.ndarray:
+        return np.repeat(np.arange(len(self.group_sizes)), self.group_sizes)
+
+    def unique_kv_bytes(self) -> int:
+        toks = int(self.group_prefix_lens.astype(np.int64).sum() + self.branch_lens.astype(np.int64).sum())
+        return toks * self.n_kv_heads * HEAD_DIM * 2 * 2
+
+    def as_single_group(self, g: int) -> AttnCase:
+        """Group g alone as an ordinary one-prefix case on the same pools (views, not copies)."""
+        b0 = int(self.group_sizes[:g].sum()); b1 = b0 + int(self.group_sizes[g])
+        shape = AttnShape(f"group{g}", n_q_heads=self.n_q_heads, n_kv_heads=self.n_kv_heads,
+                          prefix_len=int(self.group_prefix_lens[g]), n_branches=b1 - b0, gamma=self.gamma,
+                          branch_lens=tuple(int(v) for v in self.branch_lens[b0:b1]))
+        return AttnCase(shape=shape, q=self.q[b0:b1], k_pages=self.k_pages, v_pages=self.v_pages,
+                        block_table=self.block_table[b0:b1], branch_lens=self.branch_lens[b0:b1],
+                        prefix_len=int(self.group_prefix_lens[g]), num_pages=self.num_pages, max_blocks=self.max_blocks)
+
+
+def make_group_case(n_q_heads: int, n_kv_heads: int, gamma: int, group_sizes, group_prefix_lens, branch_lens,
+                    seed: int, permute_pages: bool = True, extra_pages: int = 0, layer: int = 0) -> GroupCase:
+    group_sizes = np.asarray(group_sizes, dtype=np.int32)
+    group_prefix_lens = np.asarray(group_prefix_lens, dtype=np.int32)
+    lens = np.asarray(branch_lens, dtype=np.int32)
+    assert len(group_sizes) == len(group_prefix_lens) and lens.shape == (int(group_sizes.sum()),)
+    assert (group_prefix_lens % PAGE == 0).all()
+    n_pre = group_prefix_lens // PAGE
+    n_priv = (lens.astype(np.int64) + PAGE - 1) // PAGE
+    used = int(n_pre.sum() + n_priv.sum())
+    num_pages = used + extra_pages
+    perm = _rng(seed, 7).permutation(num_pages).astype(np.int32) if permute_pages else np.arange(num_pages, dtype=np.int32)
+    group = np.repeat(np.arange(len(group_sizes)), group_sizes)
+    max_blocks = int((n_pre[group] + n_priv).max())
+    bt = np.full((len(lens), max_blocks), -1, dtype=np.int32)
+    cursor, b = 0, 0
+    for g, size in enumerate(group_sizes):
+        shared = perm[cursor:cursor + n_pre[g]]
+        cursor += int(n_pre[g])
+        for _ in range(int(size)):
+            bt[b, :n_pre[g]] = shared
+            nb = int(n_priv[b])
+            bt[b, n_pre[g]:n_pre[g] + nb] = perm[cursor:cursor + nb]
+            cursor += nb
+            b += 1
+    rng = _rng(seed + 1000003 * layer, 1)
+    q = _normal_bf16(rng, (len(lens), gamma + 1, n_q_heads, HEAD_DIM))
+    k = _normal_bf16(rng, (num_pages, n_kv_heads, PAGE, HEAD_DIM))
+    v = _normal_bf16(rng, (num_pages, n_kv_heads, PAGE, HEAD_DIM))
+    return GroupCase(n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, gamma=gamma, group_sizes=group_sizes,
+                     group_prefix_lens=group_prefix_lens, q=q, k_pages=k, v_pages=v, block_table=bt,
+                     branch_lens=lens.copy(), num_pages=num_pages, max_blocks=max_blocks)
+
+
+def poison_unused_slots_groups(case: GroupCase, bits: int = 0x7FC0) -> None:
+    """As poison_unused_slots, for a case with several prefix groups."""
+    used = np.zeros((case.num_pages, PAGE), dtype=bool)
+    group = case.group_of_branch()
+    for b in range(case.n_branches):
+        n_pre = int(case.group_prefix_lens[group[b]]) // PAGE
+        used[case.block_table[b, :n_pre], :] = True
+        L = int(case.branch_lens[b])
+        for j in range((L + PAGE - 1) // PAGE):
+            used[case.block_table[b, n_pre + j], :min(PAGE, L - j * PAGE)] = True
+    for arr in (case.k_pages, case.v_pages):
+        arr.transpose(0, 2, 1, 3)[~used] = np.uint16(bits)
+
+
+# --------------------------------------------------------------------------- #
 # draft token trees (tree verification)
 # --------------------------------------------------------------------------- #
 def make_tree_parents(n_branches: int, n_nodes: int, max_depth: int, seed: int) -> np.ndarray:
