@@ -139,6 +139,26 @@ TTS_API int tts_attn_plan(tts_ctx* ctx, const int32_t* block_table, int prefix_l
 TTS_API int tts_attn_plan_drop(tts_ctx* ctx);
 
 /*
+ * Several questions in one call (the multi-request setting of the paper's appendix: #Req questions in
+ * flight, each with B branches that share that question's prompt; Section 3.3: the forward pass turns
+ * compute-bound as B * (gamma+1) * #Req grows).  The branches are numbered group by group: group g holds
+ * group_sizes[g] consecutive branches whose block-table rows start with the same group_prefix_len[g] / 16
+ * pages.  The result for every branch is what tts_verify_attn gives for its group alone; one launch
+ * serves all groups, each shared prefix being read once per group.
+ *   group_sizes, group_prefix_len   host  [n_groups] i32, sizes >= 1 summing to n_branches, prefix
+ *                                         lengths multiples of 16 (0 allowed); n_groups <= 64
+ *   everything else as for tts_verify_attn (causal mask).  tts_attn_plan_groups is tts_attn_plan for such
+ *   calls; the kept plan also records the group arrays' contents.
+ */
+TTS_API int tts_verify_attn_groups(tts_ctx* ctx, const void* q, const void* k_pages, const void* v_pages,
+                           const int32_t* block_table, const int32_t* group_sizes,
+                           const int32_t* group_prefix_len, int n_groups, const int32_t* branch_lens,
+                           int n_branches, int gamma, void* out);
+TTS_API int tts_attn_plan_groups(tts_ctx* ctx, const int32_t* block_table, const int32_t* group_sizes,
+                         const int32_t* group_prefix_len, int n_groups, const int32_t* branch_lens,
+                         int n_branches, int rows_per_branch);
+
+/*
  * Tree verification (draft token trees, as produced by tree drafters such as the EAGLE-3 draft
  * model used in Section 4.1): the last n_nodes private tokens of each branch are tree nodes;
  * row i sees the prefix, the private tokens before the tree, itself and its ancestors.

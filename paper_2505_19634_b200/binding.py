@@ -21,7 +21,7 @@ ATTN_AUTO, ATTN_SIMT, ATTN_TCGEN05, ATTN_TCGEN05_TOKEN_MAJOR, ATTN_TCGEN05_ROW_M
 
 EXPORTED_SYMBOLS = (
     "tts_create", "tts_destroy", "tts_set_stream", "tts_verify_attn", "tts_verify_attn_tree", "tts_attn_plan",
-    "tts_attn_plan_drop",
+    "tts_attn_plan_drop", "tts_verify_attn_groups", "tts_attn_plan_groups",
     "tts_accept", "tts_accept_logits", "tts_verify_step_host_logits", "tts_majority_vote", "tts_confidence_max", "tts_greedy_search", "tts_grid_search", "tts_last_status",
     "tts_last_cuda_error", "tts_launch_count", "tts_strerror", "tts_verify_step_host",
     "tts_profile_enable", "tts_profile_read", "tts_debug_wait_timeout", "tts_verify_attn_noalloc", "tts_kv_append", "tts_kv_rollback", "tts_accept_tree",
@@ -74,6 +74,8 @@ def load_library() -> ctypes.CDLL:
     lib.tts_verify_attn_tree.argtypes = [vp, vp, vp, vp, vp, c_int, vp, vp, c_int, c_int, vp]
     lib.tts_attn_plan.argtypes = [vp, vp, c_int, vp, c_int, c_int]
     lib.tts_attn_plan_drop.argtypes = [vp]
+    lib.tts_verify_attn_groups.argtypes = [vp, vp, vp, vp, vp, ip, ip, c_int, vp, c_int, c_int, vp]
+    lib.tts_attn_plan_groups.argtypes = [vp, vp, ip, ip, c_int, vp, c_int, c_int]
     lib.tts_accept.argtypes = [vp, vp, vp, vp, vp, c_int, c_int, c_int, vp, vp]
     lib.tts_accept_logits.argtypes = [vp, vp, vp, c_int, vp, vp, c_int, c_int, c_int, vp, vp]
     lib.tts_verify_step_host_logits.argtypes = [vp, c_int, vp, POINTER(c_void_p), POINTER(c_void_p), vp, c_int, vp,
@@ -182,6 +184,24 @@ class TtsContext:
     def tts_attn_plan(self, block_table, prefix_len: int, branch_lens, n_branches: int, rows_per_branch: int):
         self._check(self._lib.tts_attn_plan(self._h, _ptr(block_table), int(prefix_len), _ptr(branch_lens),
                                             int(n_branches), int(rows_per_branch)), "tts_attn_plan")
+
+    @staticmethod
+    def _host_i32(values):
+        return (c_int32 * len(values))(*[int(v) for v in values])
+
+    def tts_verify_attn_groups(self, q, k_pages, v_pages, block_table, group_sizes, group_prefix_len, branch_lens,
+                               n_branches: int, gamma: int, out):
+        """group_sizes and group_prefix_len are host sequences of equal length."""
+        self._check(self._lib.tts_verify_attn_groups(self._h, _ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(block_table),
+                                                     self._host_i32(group_sizes), self._host_i32(group_prefix_len),
+                                                     len(group_sizes), _ptr(branch_lens), int(n_branches), int(gamma),
+                                                     _ptr(out)), "tts_verify_attn_groups")
+
+    def tts_attn_plan_groups(self, block_table, group_sizes, group_prefix_len, branch_lens, n_branches: int,
+                             rows_per_branch: int):
+        self._check(self._lib.tts_attn_plan_groups(self._h, _ptr(block_table), self._host_i32(group_sizes),
+                                                   self._host_i32(group_prefix_len), len(group_sizes), _ptr(branch_lens),
+                                                   int(n_branches), int(rows_per_branch)), "tts_attn_plan_groups")
 
     def tts_attn_plan_drop(self):
         self._check(self._lib.tts_attn_plan_drop(self._h), "tts_attn_plan_drop")

@@ -12,33 +12,40 @@ namespace tts {
 constexpr int kMaxPrivBlocks = 2, kMaxPreBlocks = 3;     // nr <= 2 row blocks
 struct GroupDesc {
     int group;                                           // b * Hkv + kvh
+    int pre_row0;                                        // stacked row of the group's first row among the rows that share its prefix
     int pre_rb0;                                         // first prefix row block of the group's stacked rows
     int priv_first[kMaxPrivBlocks], priv_n[kMaxPrivBlocks];
     int pre_first[kMaxPreBlocks], pre_n[kMaxPreBlocks];
 };
 
-// One entry of the descriptor of group (b, kvh), so that the entries can be computed by different
-// threads: e < kMaxPrivBlocks is private row block e, the others prefix row block e - kMaxPrivBlocks
-// of the group's stacked rows (tpc = tiles per CTA of the kernel that produced the pieces).
-__device__ inline void group_describe_entry(const AttnParams& p, const int* cum, int tpc, int b, int kvh, int e, GroupDesc& d) {
+// Where a set of branches that share one prefix (p describes them alone: N, P, branch_lens and the
+// segment counts are theirs) sits within a call that carries several such sets: its first branch, the tiles
+// of the sets before it in the tile list, and the prefix partial-result slots they take.
+struct SetOffsets { int first_branch, tile_off, pre_slot_base; };
+
+// One entry of the descriptor of group (b, kvh), b counted within its set, so that the entries can be
+// computed by different threads: e < kMaxPrivBlocks is private row block e, the others prefix row block
+// e - kMaxPrivBlocks of the group's stacked rows (tpc = tiles per CTA of the kernel that produced the pieces).
+__device__ inline void group_describe_entry(const AttnParams& p, const int* cum, int tpc, int b, int kvh, int e, GroupDesc& d,
+                                            const SetOffsets so = SetOffsets{0, 0, 0}) {
     const int group = b * p.Hkv + kvh;
     if (e < kMaxPrivBlocks) {
         const int rb = e, tiles_b = cum[b + 1] - cum[b];
         d.priv_first[rb] = 0; d.priv_n[rb] = 0;
         if (rb < p.n_rb_priv && tiles_b > 0) {
-            const int tb = group_tile_begin(p, cum, group) + rb * tiles_b, c0 = fast_div(tb, tpc);
-            d.priv_first[rb] = group * p.n_rb_priv + rb + c0;
+            const int tb = so.tile_off + group_tile_begin(p, cum, group) + rb * tiles_b, c0 = fast_div(tb, tpc);
+            d.priv_first[rb] = (so.first_branch * p.Hkv + group) * p.n_rb_priv + rb + c0;
             d.priv_n[rb] = fast_div(tb + tiles_b - 1, tpc) - c0 + 1;
         }
     } else {
         const int k = e - kMaxPrivBlocks;
         const int rb0 = fast_div(b * p.nr, p.rb_rows), rb_last = fast_div(b * p.nr + p.nr - 1, p.rb_rows);
-        if (k == 0) { d.group = group; d.pre_rb0 = rb0; }
+        if (k == 0) { d.group = so.first_branch * p.Hkv + group; d.pre_row0 = b * p.nr; d.pre_rb0 = rb0; }
         d.pre_first[k] = 0; d.pre_n[k] = 0;
         if (p.n_pre > 0 && rb0 + k <= rb_last) {
             const int seg = kvh * p.n_rb_pre + rb0 + k;
-            const int tb = prefix_segment_tile_begin(p, cum, seg), c0 = fast_div(tb, tpc);
-            d.pre_first[k] = seg + c0;
+            const int tb = so.tile_off + prefix_segment_tile_begin(p, cum, seg), c0 = fast_div(tb, tpc);
+            d.pre_first[k] = so.pre_slot_base + seg + c0;
             d.pre_n[k] = fast_div(tb + p.tiles_pre - 1, tpc) - c0 + 1;
         }
     }
@@ -54,7 +61,7 @@ __device__ inline void merge_group(const AttnParams& p, const GroupDesc& d, int 
     for (int r = tid >> 4; r < p.nr; r += n_threads >> 4) {
         const int i = r / p.G, gq = r - i * p.G;
         const int rb = r / p.rb_rows, r_in = r - rb * p.rb_rows;         // private row block, row within it
-        const int pr = b * p.nr + r;
+        const int pr = d.pre_row0 + r;
         const int k = pr / p.rb_rows - d.pre_rb0, pr_in = pr % p.rb_rows;   // prefix row block (relative), row within it
         const int n_pre = d.pre_n[k], np = n_pre + d.priv_n[rb];
         float m_run = -INFINITY, l_run = 0.f;

@@ -38,8 +38,8 @@ struct __align__(16) CtaPlan {
 };
 static_assert(sizeof(CtaPlan) == 512, "CtaPlan is copied as 32 x 16 bytes");
 
-// Builds the tables for the schedule `p` describes (p.plan_cta, p.plan_pieces, p.group_desc must point to
-// the context's tables).  One launch of one CTA.
-cudaError_t launch_attn_plan(const AttnParams& p, cudaStream_t st);
+// Builds the tables for the schedule that `p` and the prefix sets describe (p.plan_cta, p.plan_pieces,
+// p.group_desc must point to the context's tables).  One launch of one CTA.
+cudaError_t launch_attn_plan(const AttnParams& p, const PrefixSets& sets, cudaStream_t st);
 
 }  // namespace tts

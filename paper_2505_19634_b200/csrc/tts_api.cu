@@ -82,41 +82,59 @@ cudaError_t alloc_workspace(Ctx* c) {
                        c->n_sms * 3, &a, &b);
         pre = a > pre ? a : pre; priv = b > priv ? b : priv;
     }
+    // several prefix sets per call (token-major kernel): up to one more prefix row block per set and KV head
+    pre += (size_t)kMaxPrefixSets * f.n_kv_heads * umma_t_rows(nr);
     cudaError_t e;
     if ((e = cudaMalloc(&c->part_o_pre, pre * kHeadDim * sizeof(float))) != cudaSuccess) return e;
     if ((e = cudaMalloc(&c->part_ml_pre, pre * sizeof(float2))) != cudaSuccess) return e;
     if ((e = cudaMalloc(&c->part_o_priv, priv * kHeadDim * sizeof(float))) != cudaSuccess) return e;
     if ((e = cudaMalloc(&c->part_ml_priv, priv * sizeof(float2))) != cudaSuccess) return e;
     c->pre_rows = pre; c->priv_rows = priv;
-    if ((e = cudaMalloc(&c->group_desc, (size_t)f.max_branches * f.n_kv_heads * 64)) != cudaSuccess) return e;   // a GroupDesc is 48 bytes
+    if ((e = cudaMalloc(&c->group_desc, (size_t)f.max_branches * f.n_kv_heads * 64)) != cudaSuccess) return e;   // a GroupDesc is at most 64 bytes
     // plan of the token-major kernel (row blocks of 32 rows): one piece per segment and one more per CTA
     const size_t rb = (size_t)umma_t_rows(nr);
     const size_t n_seg = (size_t)f.max_branches * f.n_kv_heads * ((nr + rb - 1) / rb) +
                          (size_t)f.n_kv_heads * (((size_t)f.max_branches * nr + rb - 1) / rb);
-    c->plan_pieces_cap = n_seg + (size_t)c->n_sms;
+    c->plan_pieces_cap = n_seg + (size_t)kMaxPrefixSets * f.n_kv_heads + (size_t)c->n_sms;
     if ((e = cudaMalloc(&c->plan_cta, (size_t)c->n_sms * sizeof(CtaPlan))) != cudaSuccess) return e;
     return cudaMalloc(&c->plan_pieces, c->plan_pieces_cap * sizeof(PieceDesc));
 }
 
 // Checks the arguments that describe the schedule of an attention call and fills the parameters that
-// depend on them (everything but q, K/V and out).
-int attn_setup(Ctx* c, const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
+// depend on them (everything but q, K/V and out).  With several prefix sets the parameters describe the call
+// as a whole (p.P, p.n_pre and p.tiles_pre are then those of the first set and only the plan uses the rest).
+int attn_setup(Ctx* c, const int32_t* block_table, const PrefixSets& sets, const int32_t* branch_lens,
                const int32_t* tree_parents, int n_branches, int rows, AttnParams* out_p, Plan* out_pl) {
     if (!c || !block_table || !branch_lens) return TTS_ERR_INVALID;
     const tts_config& f = c->cfg;
     if (n_branches < 1 || n_branches > f.max_branches) return TTS_ERR_INVALID;
     if (rows < 1 || rows > f.max_rows_per_branch) return TTS_ERR_INVALID;
     if (rows > kMaxTreeRows) return TTS_ERR_UNSUPPORTED;
-    if (prefix_len < 0 || prefix_len % f.page_size != 0) return TTS_ERR_INVALID;
-    if (prefix_len / f.page_size > f.max_blocks_per_branch) return TTS_ERR_INVALID;
+    if (sets.n_sets < 1 || sets.n_sets > kMaxPrefixSets || sets.first_branch[0] != 0 || sets.first_branch[sets.n_sets] != n_branches)
+        return TTS_ERR_INVALID;
+    int max_set = 0;
+    for (int s = 0; s < sets.n_sets; ++s) {
+        const int prefix_len = sets.prefix_len[s], size = sets.first_branch[s + 1] - sets.first_branch[s];
+        if (size < 1) return TTS_ERR_INVALID;
+        if (prefix_len < 0 || prefix_len % f.page_size != 0) return TTS_ERR_INVALID;
+        if (prefix_len / f.page_size > f.max_blocks_per_branch) return TTS_ERR_INVALID;
+        max_set = size > max_set ? size : max_set;
+    }
     if ((reinterpret_cast<uintptr_t>(block_table) & 3u) || (reinterpret_cast<uintptr_t>(branch_lens) & 3u)) return TTS_ERR_INVALID;
 
     const int G = f.n_q_heads / f.n_kv_heads;
     const int nr = rows * G;
     const Plan pl = make_plan(c, nr, n_branches);
+    const int pre_stride = pl.copies_pre * (max_set * nr < pl.rb_rows ? max_set * nr : pl.rb_rows);
     {
+        // prefix partial results: one slot per prefix segment of every set and one more per CTA
+        long n_pre_seg = 0;
+        for (int s = 0; s < sets.n_sets; ++s)
+            if (sets.prefix_len[s] > 0)
+                n_pre_seg += (long)f.n_kv_heads * (((long)(sets.first_branch[s + 1] - sets.first_branch[s]) * nr + pl.rb_rows - 1) / pl.rb_rows);
         size_t need_pre, need_priv;
         workspace_rows(n_branches, f.n_kv_heads, nr, pl.rb_rows, pl.copies, pl.copies_pre, pl.grid, &need_pre, &need_priv);
+        need_pre = (size_t)(n_pre_seg + pl.grid) * pre_stride;
         if (need_pre > c->pre_rows || need_priv > c->priv_rows) return TTS_ERR_INVALID;
     }
     AttnParams& p = *out_p;
@@ -128,17 +146,17 @@ int attn_setup(Ctx* c, const int32_t* block_table, int prefix_len, const int32_t
     // the token-major kernel and its merge kernel run from the plan tables
     if (pl.impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR) { p.group_desc = c->group_desc; p.plan_cta = c->plan_cta; p.plan_pieces = c->plan_pieces; }
     p.N = n_branches; p.R = rows; p.Hq = f.n_q_heads; p.Hkv = f.n_kv_heads; p.G = G; p.nr = nr;
-    p.P = prefix_len; p.max_blocks = f.max_blocks_per_branch; p.num_pages = f.num_pages;
+    p.P = sets.prefix_len[0]; p.max_blocks = f.max_blocks_per_branch; p.num_pages = f.num_pages;
     p.rb_rows = pl.rb_rows;
-    p.pre_stride = pl.copies_pre * (n_branches * nr < pl.rb_rows ? n_branches * nr : pl.rb_rows);
+    p.pre_stride = pre_stride;
     p.priv_stride = pl.copies * (nr < pl.rb_rows ? nr : pl.rb_rows);
     p.copies = pl.copies; p.copies_pre = pl.copies_pre;
     p.n_rb_pre = ceil_div(n_branches * nr, pl.rb_rows);
     p.n_rb_priv = ceil_div(nr, pl.rb_rows);
-    p.n_pre = prefix_len > 0 ? f.n_kv_heads * p.n_rb_pre : 0;
-    if ((long long)n_branches * f.n_kv_heads * p.n_pre >= (1ll << 31)) return TTS_ERR_UNSUPPORTED;
+    p.n_pre = p.P > 0 ? f.n_kv_heads * p.n_rb_pre : 0;
+    if ((long long)n_branches * f.n_kv_heads * f.n_kv_heads * p.n_rb_pre >= (1ll << 31)) return TTS_ERR_UNSUPPORTED;
     p.tile_tokens = pl.tile_tokens;
-    p.tiles_pre = ceil_div(prefix_len, pl.tile_tokens);
+    p.tiles_pre = ceil_div(p.P, pl.tile_tokens);
     p.grid = pl.grid;
     p.out_dtype = f.out_dtype; p.debug = f.debug_bounds;
     const float scale = f.softmax_scale > 0.f ? f.softmax_scale : 1.0f / sqrtf((float)f.head_dim);
@@ -147,31 +165,74 @@ int attn_setup(Ctx* c, const int32_t* block_table, int prefix_len, const int32_t
     return TTS_OK;
 }
 
+PrefixSets one_set(int prefix_len, int n_branches) {
+    PrefixSets sets;
+    memset(&sets, 0, sizeof sets);
+    sets.n_sets = 1; sets.first_branch[1] = n_branches; sets.prefix_len[0] = prefix_len;
+    return sets;
+}
+
+// group_sizes / group_prefix_len (host arrays) as prefix sets; false when they are not a valid description
+bool sets_from_groups(const int32_t* group_sizes, const int32_t* group_prefix_len, int n_groups, int n_branches, PrefixSets* sets) {
+    if (!group_sizes || !group_prefix_len || n_groups < 1 || n_groups > kMaxPrefixSets) return false;
+    memset(sets, 0, sizeof *sets);
+    sets->n_sets = n_groups;
+    long first = 0;
+    for (int g = 0; g < n_groups; ++g) {
+        if (group_sizes[g] < 1) return false;
+        sets->first_branch[g] = (int)first;
+        sets->prefix_len[g] = group_prefix_len[g];
+        first += group_sizes[g];
+        if (first > n_branches) return false;
+    }
+    sets->first_branch[n_groups] = (int)first;
+    return first == n_branches;
+}
+
+bool same_sets(const PrefixSets& a, const PrefixSets& b) {
+    return a.n_sets == b.n_sets && memcmp(a.first_branch, b.first_branch, sizeof(int) * (a.n_sets + 1)) == 0 &&
+           memcmp(a.prefix_len, b.prefix_len, sizeof(int) * a.n_sets) == 0;
+}
+
 // Does the plan in the context's tables, built by tts_attn_plan, describe this call?
-bool plan_matches(const Ctx* c, const int32_t* block_table, int prefix_len, const int32_t* branch_lens, int n_branches, int rows) {
+bool plan_matches(const Ctx* c, const int32_t* block_table, const PrefixSets& sets, const int32_t* branch_lens, int n_branches, int rows) {
     return c->plan_explicit && c->plan_key.block_table == block_table && c->plan_key.branch_lens == branch_lens &&
-           c->plan_key.prefix_len == prefix_len && c->plan_key.n_branches == n_branches && c->plan_key.rows == rows;
+           c->plan_key.n_branches == n_branches && c->plan_key.rows == rows && same_sets(c->plan_key.sets, sets);
 }
 
 int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
-                const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
+                const int32_t* block_table, const PrefixSets& sets, const int32_t* branch_lens,
                 const int32_t* tree_parents, int n_branches, int rows, void* out) {
     if (!c || !q || !k_pages || !v_pages || !out) return TTS_ERR_INVALID;
     if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(out)) return TTS_ERR_INVALID;
     AttnParams p;
     Plan pl;
-    const int rc = attn_setup(c, block_table, prefix_len, branch_lens, tree_parents, n_branches, rows, &p, &pl);
+    const int rc = attn_setup(c, block_table, sets, branch_lens, tree_parents, n_branches, rows, &p, &pl);
     if (rc != TTS_OK) return rc;
+    if (sets.n_sets > 1 && pl.impl != TTS_ATTN_TCGEN05_TOKEN_MAJOR) {
+        // the other kernels take one prefix per launch: set by set, on the rows, table rows and lengths of each
+        const size_t row_elts = (size_t)rows * c->cfg.n_q_heads * kHeadDim;
+        const size_t out_elt = c->cfg.out_dtype == TTS_OUT_FP32 ? 4 : 2;
+        for (int s = 0; s < sets.n_sets; ++s) {
+            const int b0 = sets.first_branch[s], n = sets.first_branch[s + 1] - b0;
+            const int rc_s = attn_common(c, static_cast<const char*>(q) + b0 * row_elts * 2, k_pages, v_pages,
+                                         block_table + (size_t)b0 * c->cfg.max_blocks_per_branch, one_set(sets.prefix_len[s], n),
+                                         branch_lens + b0, tree_parents ? tree_parents + (size_t)b0 * rows : nullptr, n, rows,
+                                         static_cast<char*>(out) + b0 * row_elts * out_elt);
+            if (rc_s != TTS_OK) return rc_s;
+        }
+        return TTS_OK;
+    }
     p.q = static_cast<const __nv_bfloat16*>(q);
     p.k_pages = static_cast<const __nv_bfloat16*>(k_pages);
     p.v_pages = static_cast<const __nv_bfloat16*>(v_pages);
     p.out = out;
     cudaError_t e;
 
-    if (pl.impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR && !plan_matches(c, block_table, prefix_len, branch_lens, n_branches, rows)) {
+    if (pl.impl == TTS_ATTN_TCGEN05_TOKEN_MAJOR && !plan_matches(c, block_table, sets, branch_lens, n_branches, rows)) {
         // no plan from tts_attn_plan for these arguments: build one for this call alone
         c->plan_explicit = 0;
-        e = launch_attn_plan(p, c->stream);
+        e = launch_attn_plan(p, sets, c->stream);
         if (e != cudaSuccess) return cuda_fail(c, e);
         c->launches += 1;
     }
@@ -200,6 +261,22 @@ int attn_common(Ctx* c, const void* q, const void* k_pages, const void* v_pages,
     if (e != cudaSuccess) return cuda_fail(c, e);
     c->launches += 1;
     if (prof) { record(ev[2]); c->prof_n += 1; }
+    return TTS_OK;
+}
+
+int plan_common(Ctx* c, const int32_t* block_table, const PrefixSets& sets, const int32_t* branch_lens, int n_branches, int rows) {
+    AttnParams p;
+    Plan pl;
+    const int rc = attn_setup(c, block_table, sets, branch_lens, nullptr, n_branches, rows, &p, &pl);
+    if (rc != TTS_OK) return rc;
+    c->plan_explicit = 0;
+    if (pl.impl != TTS_ATTN_TCGEN05_TOKEN_MAJOR) return TTS_OK;      // the other kernels derive their schedule themselves
+    const cudaError_t e = launch_attn_plan(p, sets, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->launches += 1;
+    c->plan_key.block_table = block_table; c->plan_key.branch_lens = branch_lens;
+    c->plan_key.n_branches = n_branches; c->plan_key.rows = rows; c->plan_key.sets = sets;
+    c->plan_explicit = 1;
     return TTS_OK;
 }
 
@@ -272,34 +349,39 @@ int tts_verify_attn(tts_ctx* ctx, const void* q, const void* k_pages, const void
     if (mask_kind == TTS_MASK_TREE) return TTS_ERR_UNSUPPORTED;     // needs parents: tts_verify_attn_tree
     if (mask_kind != TTS_MASK_CAUSAL) return TTS_ERR_UNSUPPORTED;
     if (gamma < 0) return TTS_ERR_INVALID;
-    return attn_common(reinterpret_cast<Ctx*>(ctx), q, k_pages, v_pages, block_table, prefix_len,
+    return attn_common(reinterpret_cast<Ctx*>(ctx), q, k_pages, v_pages, block_table, one_set(prefix_len, n_branches),
                        branch_lens, nullptr, n_branches, gamma + 1, out);
+}
+
+int tts_verify_attn_groups(tts_ctx* ctx, const void* q, const void* k_pages, const void* v_pages,
+                           const int32_t* block_table, const int32_t* group_sizes, const int32_t* group_prefix_len,
+                           int n_groups, const int32_t* branch_lens, int n_branches, int gamma, void* out) {
+    PrefixSets sets;
+    if (gamma < 0 || !sets_from_groups(group_sizes, group_prefix_len, n_groups, n_branches, &sets)) return TTS_ERR_INVALID;
+    return attn_common(reinterpret_cast<Ctx*>(ctx), q, k_pages, v_pages, block_table, sets, branch_lens, nullptr,
+                       n_branches, gamma + 1, out);
 }
 
 int tts_verify_attn_tree(tts_ctx* ctx, const void* q, const void* k_pages, const void* v_pages,
                          const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
                          const int32_t* tree_parents, int n_branches, int n_nodes, void* out) {
     if (!tree_parents) return TTS_ERR_INVALID;
-    return attn_common(reinterpret_cast<Ctx*>(ctx), q, k_pages, v_pages, block_table, prefix_len,
+    return attn_common(reinterpret_cast<Ctx*>(ctx), q, k_pages, v_pages, block_table, one_set(prefix_len, n_branches),
                        branch_lens, tree_parents, n_branches, n_nodes, out);
 }
 
 int tts_attn_plan(tts_ctx* ctx, const int32_t* block_table, int prefix_len, const int32_t* branch_lens,
                   int n_branches, int rows_per_branch) {
-    Ctx* c = reinterpret_cast<Ctx*>(ctx);
-    AttnParams p;
-    Plan pl;
-    const int rc = attn_setup(c, block_table, prefix_len, branch_lens, nullptr, n_branches, rows_per_branch, &p, &pl);
-    if (rc != TTS_OK) return rc;
-    c->plan_explicit = 0;
-    if (pl.impl != TTS_ATTN_TCGEN05_TOKEN_MAJOR) return TTS_OK;      // the other kernels derive their schedule themselves
-    const cudaError_t e = launch_attn_plan(p, c->stream);
-    if (e != cudaSuccess) return cuda_fail(c, e);
-    c->launches += 1;
-    c->plan_key.block_table = block_table; c->plan_key.branch_lens = branch_lens;
-    c->plan_key.prefix_len = prefix_len; c->plan_key.n_branches = n_branches; c->plan_key.rows = rows_per_branch;
-    c->plan_explicit = 1;
-    return TTS_OK;
+    return plan_common(reinterpret_cast<Ctx*>(ctx), block_table, one_set(prefix_len, n_branches), branch_lens, n_branches,
+                       rows_per_branch);
+}
+
+int tts_attn_plan_groups(tts_ctx* ctx, const int32_t* block_table, const int32_t* group_sizes,
+                         const int32_t* group_prefix_len, int n_groups, const int32_t* branch_lens, int n_branches,
+                         int rows_per_branch) {
+    PrefixSets sets;
+    if (!sets_from_groups(group_sizes, group_prefix_len, n_groups, n_branches, &sets)) return TTS_ERR_INVALID;
+    return plan_common(reinterpret_cast<Ctx*>(ctx), block_table, sets, branch_lens, n_branches, rows_per_branch);
 }
 
 int tts_attn_plan_drop(tts_ctx* ctx) {

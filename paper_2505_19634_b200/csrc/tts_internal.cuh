@@ -32,6 +32,15 @@ constexpr int kMaxBranches = 1024;
 // workspace.
 struct CtaPlan;
 struct PieceDesc;
+
+// Sets of branches that share a prefix each (several questions in one call): set s holds the branches
+// [first_branch[s], first_branch[s + 1]) and its prefix is prefix_len[s] tokens long.
+constexpr int kMaxPrefixSets = 64;
+struct PrefixSets {
+    int n_sets;
+    int first_branch[kMaxPrefixSets + 1];
+    int prefix_len[kMaxPrefixSets];
+};
 struct AttnParams {
     const __nv_bfloat16* q;
     const __nv_bfloat16* k_pages;
@@ -297,7 +306,7 @@ struct Ctx {
     // plan of the token-major kernel (attn_plan.cuh): one record per CTA, the list of all pieces
     CtaPlan* plan_cta; PieceDesc* plan_pieces; size_t plan_pieces_cap;
     // the arguments the plan in the tables was built from by tts_attn_plan (valid while plan_explicit is set)
-    struct { const int32_t* block_table; const int32_t* branch_lens; int prefix_len, n_branches, rows; } plan_key;
+    struct { const int32_t* block_table; const int32_t* branch_lens; int n_branches, rows; PrefixSets sets; } plan_key;
     int plan_explicit;
     // staging for the host entry point
     void* stage; size_t stage_bytes;
