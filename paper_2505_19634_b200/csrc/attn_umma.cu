@@ -5,23 +5,21 @@
 // 128 KV tokens of one KV head = 8 pages gathered through the block table, each page-head tile
 // (16 tokens x 128 dims, 4 KiB contiguous) arriving as two 128-byte-swizzled TMA boxes.
 //
-//   warp 4      producer: per tile, arms the K and V "full" barriers with the byte count and
+//   warp 8      producer: per tile, arms the K and V "full" barriers with the byte count and
 //               issues the TMA boxes (K ring and V ring, 2 slots x 32 KiB each)
-//   warp 5      MMA issuer (one thread): S = Q K^T into one of two TMEM buffers, then
+//   warp 9      MMA issuer (one thread): S = Q K^T into one of two TMEM buffers, then
 //               O (+)= P V once the softmax warps have published P; frees ring slots with
 //               tcgen05.commit
-//   warps 0-3   softmax: thread = TMEM lane = query row.  Reads S, keeps the running max m and
-//               sum l in fp32, writes P (bf16, swizzled K-major) to shared memory for the second
-//               contraction, rescales O in TMEM only when the max moved by more than 2^8
-//               (the final result is exact either way, l carries the same reference), and
-//               writes the piece's partial (m, l, O) at the end.
+//   warps 0-7   softmax: two threads per query row (TMEM lane), each on one half of the tile's 128 key
+//               columns.  A thread reads its 64 scores once, the pair agrees on the row maximum
+//               through shared memory, and each writes its half of the row of P (bf16, swizzled
+//               K-major) for the second contraction.  O is rescaled in TMEM only when the max moved
+//               by more than 2^8 (the final result is exact either way, l carries the same
+//               reference); each thread keeps the sum of its own columns; the piece's partial
+//               (m, l, O) is written at the end.
 //
-// Few query rows per KV head (nr = (gamma+1) * G, e.g. 20) would leave most of the 128-row MMA
-// tile idle, so the rows of a private segment are replicated `copies` = 2 or 4 times along M and
-// copy c only looks at its own 128/copies-column slice of every S tile: the softmax work per
-// thread shrinks by `copies`, no cross-thread reduction is needed (each copy is an independent
-// split of the keys with its own m and l), and the merge kernel folds the copies together with
-// the pieces.  The MMA cost is unchanged (M is 128 regardless).
+// This is the kernel for many query rows per KV head (draft trees: nodes x GQA group rows); with few rows
+// most of the 128-row tile is padding and the token-major kernel (attn_umma_t.cu) is the one to use.
 //
 // Every wait is bounded: when a limit runs out the CTA raises TTS_ERR_DEVICE_TIMEOUT in the
 // status word, all roles leave their loops, in-flight copies are awaited (bounded) and TMEM is
@@ -41,7 +39,9 @@ using namespace ptx;
 
 constexpr int kTile = kUmmaTileTokens;            // 128 tokens
 constexpr int kRows = kUmmaRows;                   // 128 = MMA M
-constexpr int kThreadsUmma = 192;
+constexpr int kSoftmaxThreads = 256;                 // 8 warps: (TMEM lane quarter, column half)
+constexpr int kThreadsUmma = kSoftmaxThreads + 64;
+constexpr int kProducerWarp = kSoftmaxThreads / 32, kMmaWarp = kProducerWarp + 1;
 constexpr int kHalfBytes = kRows * 128;            // one 64-element K-block of a 128-row operand: 16 KiB
 constexpr int kOperandBytes = 2 * kHalfBytes;      // 32 KiB
 constexpr int kRing = 2;
@@ -55,7 +55,8 @@ constexpr int kOffV = kOffK + kRing * kOperandBytes;
 constexpr int kOffBar = kOffV + kRing * kOperandBytes;        // 196608
 constexpr int kNumBars = 16;
 constexpr int kOffMisc = kOffBar + kNumBars * 8;
-constexpr int kOffCum = kOffMisc + 64;
+constexpr int kOffXch = kOffMisc + 64;                         // float[5][128]: row maxima of two tiles x two halves, row sums
+constexpr int kOffCum = kOffXch + 5 * kRows * 4;
 constexpr int kUmmaMaxBranches = 1024;
 constexpr int kSmemBytes = kOffCum + (kUmmaMaxBranches + 1) * 4 + 1024;   // + slack for manual alignment
 
@@ -102,12 +103,12 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
         for (int i = 0; i < kRing; ++i) {
             mbar_init(bar(K_FULL + i), 1); mbar_init(bar(K_EMPTY + i), 1);
             mbar_init(bar(V_FULL + i), 1); mbar_init(bar(V_EMPTY + i), 1);
-            mbar_init(bar(S_FULL + i), 1); mbar_init(bar(S_FREE + i), 128);
+            mbar_init(bar(S_FULL + i), 1); mbar_init(bar(S_FREE + i), kSoftmaxThreads);
         }
-        mbar_init(bar(P_FULL), 128); mbar_init(bar(PV_DONE), 1); mbar_init(bar(Q_FULL), 128);
+        mbar_init(bar(P_FULL), kSoftmaxThreads); mbar_init(bar(PV_DONE), 1); mbar_init(bar(Q_FULL), kSoftmaxThreads);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 5) {
+    if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + kOffMisc + 4), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -119,7 +120,7 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
     const uint32_t tmem_s[2] = {tmem, tmem + 128u};
     const uint32_t tmem_o = tmem + 256u;
 
-    if (warp == 4) {
+    if (warp == kProducerWarp) {
         // =========================== producer ===========================
         int it = 0;                                         // tiles issued by this CTA
         int g = g_begin;
@@ -174,7 +175,7 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 mbar_wait(bar(V_FULL + j % kRing), (j / kRing) & 1, quiet);
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kMmaWarp) {
         // =========================== MMA issuer ===========================
         if (lane == 0) {
             constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
@@ -227,46 +228,42 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
         }
     } else {
         // =========================== softmax warps ===========================
-        const int L = tid;                                  // TMEM lane = row of the MMA tile
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const int quarter = warp & 3, half = warp >> 2;     // TMEM lane quarter of this warp; column half of this thread
+        const int L = quarter * 32 + lane;                  // TMEM lane = row of the MMA tile
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        constexpr int W = kTile / 2;                        // S columns (keys) this thread looks at
+        const int col0 = half * W;
+        float* xch = reinterpret_cast<float*>(smem + kOffXch);   // [2 tile parities][2 halves][128 rows]
         int it = 0;
         int g = g_begin;
         bool alive = true;
         while (g < g_end && alive) {
             const SegInfo seg = segment_of_tile(p, cum, g);
             const int t_first = g - seg.tile_begin, t_last = min(seg.n_tiles, g_end - seg.tile_begin);
-            const int ncopy = seg.kind == 0 ? 1 : p.copies;
-            const int rpc = kRows / ncopy;                   // TMEM lanes per copy
-            const int W = kTile / ncopy;                     // S columns this thread looks at
-            const int copy = L / rpc, r = L % rpc;
-            const bool valid = r < seg.n_rows;
-            const int col0 = copy * W;
+            const bool valid = L < seg.n_rows;
 
-            // ---- stage Q (replicated per copy, zero rows elsewhere), per-row mask ----
+            // ---- stage Q (each thread half of its row, zero rows past the block), per-row mask ----
             unsigned long long vis = ~0ull;
             {
                 const __nv_bfloat16* src = nullptr;
                 if (valid) {
-                    int row = seg.row0 + r, b = seg.b;
+                    int row = seg.row0 + L, b = seg.b;
                     if (seg.kind == 0) { b = row / p.nr; row = row % p.nr; }
                     const int i = row / p.G, gq = row % p.G;
                     src = p.q + (((size_t)b * p.R + i) * p.Hq + seg.kvh * p.G + gq) * kHeadDim;
                     if (seg.kind == 1) vis = row_visibility(p, b, i);
                 }
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
+                for (int c = 8 * half; c < 8 * half + 8; ++c) {
                     uint4 v = make_uint4(0, 0, 0, 0);
                     if (valid) v = __ldg(reinterpret_cast<const uint4*>(src) + c);
                     *reinterpret_cast<uint4*>(smem + kOffQ + kmajor_chunk_off(L, c)) = v;
-                    // a copy only ever writes its own column slice of its P row: the rest must be zero
-                    // (the previous piece's last P.V has completed, see the piece epilogue)
-                    if (ncopy > 1) *reinterpret_cast<uint4*>(smem + kOffP + kmajor_chunk_off(L, c)) = make_uint4(0, 0, 0, 0);
                 }
             }
             fence_proxy_async();
             mbar_arrive(bar(Q_FULL));
 
-            float m_ref = -INFINITY, l_sum = 0.f;           // reference max (log2 units) and running sum
+            float m_ref = -INFINITY, l_sum = 0.f;           // reference max (log2 units); sum over this thread's columns
             const int Ltok = seg.n_tokens;
             const int tail0 = seg.kind == 1 ? Ltok - p.R : Ltok;     // first token that needs the row mask
 
@@ -277,31 +274,30 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 alive = __all_sync(0xffffffffu, mbar_wait(bar(S_FULL + sb), (it >> 1) & 1, ab));
                 if (!alive) break;
                 tc_fence_after();
-                const uint32_t s_addr = tmem_s[sb] + lane_base + (uint32_t)col0;
 
-                auto allowed = [&](int col) -> bool {       // col = column inside the tile
-                    const int j = tok0 + col;
-                    if (j >= Ltok) return false;
-                    if (j >= tail0) return (vis >> (j - tail0)) & 1ull;
-                    return true;
-                };
-
-                // pass 1: row max over this thread's columns
-                float mx = -INFINITY;
-                for (int ch = 0; ch < W / 32; ++ch) {
-                    uint32_t sv[32];
-                    tmem_ld32(s_addr + 32u * ch, sv);
-                    tmem_wait_ld();
-                    if (need_mask) {
+                // this thread's 64 scores, read once; masked ones become -inf
+                float sv[W];
+                tmem_ld32(tmem_s[sb] + lane_base + (uint32_t)col0, reinterpret_cast<uint32_t*>(sv));
+                tmem_ld32(tmem_s[sb] + lane_base + (uint32_t)col0 + 32u, reinterpret_cast<uint32_t*>(sv) + 32);
+                tmem_wait_ld();
+                tc_fence_before();
+                mbar_arrive(bar(S_FREE + sb));               // the scores are in registers: S may be overwritten
+                if (need_mask) {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            if (allowed(col0 + 32 * ch + c)) mx = fmaxf(mx, __uint_as_float(sv[c]));
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(sv[c]));
+                    for (int c = 0; c < W; ++c) {
+                        const int j = tok0 + col0 + c;
+                        const bool ok = j < Ltok && (j < tail0 || ((vis >> (j - tail0)) & 1ull));
+                        if (!ok) sv[c] = -INFINITY;
                     }
                 }
-                mx *= p.scale_log2;                          // scale > 0; -inf stays -inf
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < W; ++c) mx = fmaxf(mx, sv[c]);
+                // the row maximum over both halves
+                float* x = xch + (it & 1) * 2 * kRows;
+                x[half * kRows + L] = mx;
+                asm volatile("barrier.cta.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");
+                mx = fmaxf(x[L], x[kRows + L]) * p.scale_log2;      // scale > 0; -inf stays -inf
                 const bool move = mx > m_ref + 8.f || (m_ref == -INFINITY && mx > -INFINITY);
                 const float m_new = move ? mx : m_ref;
                 const float factor = (move && m_ref != -INFINITY) ? ex2(m_ref - m_new) : 1.f;
@@ -312,49 +308,37 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                     if (!alive) break;
                     tc_fence_after();
                 }
-                if (t > t_first && __any_sync(0xffffffffu, factor != 1.f)) {
-                    for (int ch = 0; ch < 4; ++ch) {
+                if (t > t_first && __any_sync(0xffffffffu, factor != 1.f)) {     // this thread's half of its O row
+                    for (int ch = 0; ch < 2; ++ch) {
                         uint32_t ov[32];
-                        tmem_ld32(tmem_o + lane_base + 32u * ch, ov);
+                        tmem_ld32(tmem_o + lane_base + (uint32_t)(col0 + 32 * ch), ov);
                         tmem_wait_ld();
 #pragma unroll
                         for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * factor);
-                        tmem_st32(tmem_o + lane_base + 32u * ch, ov);
+                        tmem_st32(tmem_o + lane_base + (uint32_t)(col0 + 32 * ch), ov);
                     }
                     tmem_wait_st();
                 }
                 l_sum *= factor;
                 m_ref = m_new;
 
-                // pass 2: probabilities -> P (bf16) in shared memory
+                // probabilities -> this thread's half of its row of P (bf16) in shared memory
                 const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-                for (int ch = 0; ch < W / 32; ++ch) {
-                    uint32_t sv[32];
-                    tmem_ld32(s_addr + 32u * ch, sv);
-                    tmem_wait_ld();
-                    float pr[32];
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        float e = ex2(fmaf(__uint_as_float(sv[c]), p.scale_log2, neg_m));
-                        if (need_mask && !allowed(col0 + 32 * ch + c)) e = 0.f;
-                        pr[c] = e;
-                        l_sum += e;
-                    }
-                    const int tc0 = col0 + 32 * ch;          // first token column of this chunk
+                for (int q8 = 0; q8 < W / 8; ++q8) {
+                    float pr[8];
 #pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        uint4 pk;
-                        __nv_bfloat162 h0 = __floats2bfloat162_rn(pr[8 * q4 + 0], pr[8 * q4 + 1]);
-                        __nv_bfloat162 h1 = __floats2bfloat162_rn(pr[8 * q4 + 2], pr[8 * q4 + 3]);
-                        __nv_bfloat162 h2 = __floats2bfloat162_rn(pr[8 * q4 + 4], pr[8 * q4 + 5]);
-                        __nv_bfloat162 h3 = __floats2bfloat162_rn(pr[8 * q4 + 6], pr[8 * q4 + 7]);
-                        pk.x = *reinterpret_cast<uint32_t*>(&h0); pk.y = *reinterpret_cast<uint32_t*>(&h1);
-                        pk.z = *reinterpret_cast<uint32_t*>(&h2); pk.w = *reinterpret_cast<uint32_t*>(&h3);
-                        *reinterpret_cast<uint4*>(smem + kOffP + kmajor_chunk_off(L, (tc0 >> 3) + q4)) = pk;
+                    for (int c = 0; c < 8; ++c) {
+                        pr[c] = ex2(fmaf(sv[8 * q8 + c], p.scale_log2, neg_m));       // masked: ex2(-inf) = 0
+                        l_sum += pr[c];
                     }
+                    uint4 pk;
+                    __nv_bfloat162 h0 = __floats2bfloat162_rn(pr[0], pr[1]), h1 = __floats2bfloat162_rn(pr[2], pr[3]);
+                    __nv_bfloat162 h2 = __floats2bfloat162_rn(pr[4], pr[5]), h3 = __floats2bfloat162_rn(pr[6], pr[7]);
+                    pk.x = *reinterpret_cast<uint32_t*>(&h0); pk.y = *reinterpret_cast<uint32_t*>(&h1);
+                    pk.z = *reinterpret_cast<uint32_t*>(&h2); pk.w = *reinterpret_cast<uint32_t*>(&h3);
+                    *reinterpret_cast<uint4*>(smem + kOffP + kmajor_chunk_off(L, (col0 >> 3) + q8)) = pk;
                 }
-                tc_fence_before();
-                mbar_arrive(bar(S_FREE + sb));               // S buffer may be overwritten
 
                 // last tile of a private segment: zero the V rows of the loaded pages past the branch end
                 if (need_mask) {
@@ -364,7 +348,7 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                         const int slot = it % kRing;
                         alive = __all_sync(0xffffffffu, mbar_wait(bar(V_FULL + slot), (it / kRing) & 1, ab));
                         if (!alive) break;
-                        for (int idx = tid; idx < (n_loaded - n_valid) * 16; idx += 128) {
+                        for (int idx = tid; idx < (n_loaded - n_valid) * 16; idx += kSoftmaxThreads) {
                             const int row = n_valid + idx / 16, c = idx % 16;
                             *reinterpret_cast<uint4*>(smem + kOffV + slot * kOperandBytes + (c >> 3) * kHalfBytes + row * 128 + ((c & 7) << 4)) =
                                 make_uint4(0, 0, 0, 0);
@@ -382,20 +366,23 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
             tc_fence_after();
             float* po; float2* pml;
             piece_slot(p, seg, blockIdx.x, po, pml);
-            const int prow = copy * seg.n_rows + r;          // copies of a private piece are stacked
-            for (int ch = 0; ch < 4; ++ch) {
+            float* lx = xch + 4 * kRows;                     // the two halves' sums of a row
+            if (half == 1) lx[L] = l_sum;
+            for (int ch = 0; ch < 2; ++ch) {
                 uint32_t ov[32];
-                tmem_ld32(tmem_o + lane_base + 32u * ch, ov);
+                tmem_ld32(tmem_o + lane_base + (uint32_t)(col0 + 32 * ch), ov);
                 tmem_wait_ld();
                 if (valid) {
-                    float4* dst = reinterpret_cast<float4*>(po + (size_t)prow * kHeadDim + 32 * ch);
+                    float4* dst = reinterpret_cast<float4*>(po + (size_t)L * kHeadDim + col0 + 32 * ch);
 #pragma unroll
                     for (int c = 0; c < 8; ++c)
                         dst[c] = make_float4(__uint_as_float(ov[4 * c]), __uint_as_float(ov[4 * c + 1]),
                                              __uint_as_float(ov[4 * c + 2]), __uint_as_float(ov[4 * c + 3]));
                 }
             }
-            if (valid) pml[prow] = make_float2(m_ref, l_sum);
+            asm volatile("barrier.cta.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");
+            if (valid && half == 0) pml[L] = make_float2(m_ref, l_sum + lx[L]);
+            asm volatile("barrier.cta.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");   // lx is free for the next piece
             tc_fence_before();
             g = seg.tile_begin + t_last;
         }
@@ -404,7 +391,7 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
     // ---- teardown: everyone arrives here, normally or after an abort ----
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == kMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
@@ -475,7 +462,7 @@ const CUtensorMap* umma_pool_map(Ctx* c, const void* pool, int kind, cudaError_t
 
 bool umma_available() { return true; }
 
-int umma_copies(int nr) { return nr <= 32 ? 4 : (nr <= 64 ? 2 : 1); }
+int umma_copies(int nr) { (void)nr; return 1; }
 
 cudaError_t launch_attn_umma(Ctx* c, const AttnParams& p, cudaStream_t st) {
     if (p.N > kUmmaMaxBranches) return cudaErrorInvalidValue;
