@@ -3,7 +3,7 @@
 //
 // One persistent CTA per SM walks its run of the global tile list (tts_internal.cuh).  A tile is
 // 128 KV tokens of one KV head = 8 pages gathered through the block table, each page-head tile
-// (16 tokens x 128 dims, 4 KiB contiguous) arriving as two 128-byte-swizzled TMA boxes.
+// (16 tokens x 128 dims, 4 KiB contiguous) arriving as one 128-byte-swizzled 5-D TMA box.
 //
 //   warp 8      producer: per tile, arms the K and V "full" barriers with the byte count and
 //               issues the TMA boxes (K ring and V ring, 2 slots x 32 KiB each)
@@ -70,6 +70,13 @@ __device__ __forceinline__ uint32_t kmajor_chunk_off(int row, int chunk) {
     return (uint32_t)((chunk >> 3) * kHalfBytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
 
+// One mbarrier arrival for the whole warp, after every lane's preceding work (arrivals of single threads
+// on one barrier serialise, so the barriers count warps).
+__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+}
+
 struct PieceWalk {                    // every role iterates the CTA's pieces the same way
     int g, g_end;
 };
@@ -103,9 +110,9 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
         for (int i = 0; i < kRing; ++i) {
             mbar_init(bar(K_FULL + i), 1); mbar_init(bar(K_EMPTY + i), 1);
             mbar_init(bar(V_FULL + i), 1); mbar_init(bar(V_EMPTY + i), 1);
-            mbar_init(bar(S_FULL + i), 1); mbar_init(bar(S_FREE + i), kSoftmaxThreads);
+            mbar_init(bar(S_FULL + i), 1); mbar_init(bar(S_FREE + i), kSoftmaxThreads / 32);
         }
-        mbar_init(bar(P_FULL), kSoftmaxThreads); mbar_init(bar(PV_DONE), 1); mbar_init(bar(Q_FULL), kSoftmaxThreads);
+        mbar_init(bar(P_FULL), kSoftmaxThreads / 32); mbar_init(bar(PV_DONE), 1); mbar_init(bar(Q_FULL), kSoftmaxThreads / 32);   // the softmax warps arrive once per warp
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMmaWarp) {
@@ -125,6 +132,7 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
         int it = 0;                                         // tiles issued by this CTA
         int g = g_begin;
         bool alive = true;
+        const uint64_t stream_once = l2_policy_evict_first();
         while (g < g_end && alive) {
             const SegInfo seg = segment_of_tile(p, cum, g);
             const int t_first = g - seg.tile_begin, t_last = min(seg.n_tiles, g_end - seg.tile_begin);
@@ -136,7 +144,9 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 const int n_pages = ceil_div(min(kTile, seg.n_tokens - tok0), kPage);
                 int page = 0;
                 if (lane < n_pages) page = checked_page(p, bt, (seg.tok_begin + tok0) / kPage + lane);
-                const int y = (page * p.Hkv + seg.kvh) * kPage;
+                // one box per page-head tile (4 KiB), laid out [token half][dim half][8 tokens][128 bytes], so the
+                // pages of a tile form one MMA operand with 2 KiB between its 8-token groups
+                const int page_head = page * p.Hkv + seg.kvh;
                 // K
                 if (lane == 0) {
                     alive = mbar_wait(bar(K_EMPTY + slot), par, ab);
@@ -144,11 +154,8 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 }
                 alive = __shfl_sync(0xffffffffu, alive, 0);
                 if (!alive) break;
-                if (lane < n_pages) {
-                    const uint32_t dst = sbase + kOffK + slot * kOperandBytes + lane * 2048;
-                    tma_load_2d(dst, &tm_k, 0, y, bar(K_FULL + slot));
-                    tma_load_2d(dst + kHalfBytes, &tm_k, 64, y, bar(K_FULL + slot));
-                }
+                if (lane < n_pages)
+                    tma_load_page(sbase + kOffK + slot * kOperandBytes + lane * 4096, &tm_k, page_head, bar(K_FULL + slot), stream_once);
                 // V
                 if (lane == 0) {
                     alive = mbar_wait(bar(V_EMPTY + slot), par, ab);
@@ -156,11 +163,8 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 }
                 alive = __shfl_sync(0xffffffffu, alive, 0);
                 if (!alive) break;
-                if (lane < n_pages) {
-                    const uint32_t dst = sbase + kOffV + slot * kOperandBytes + lane * 2048;
-                    tma_load_2d(dst, &tm_v, 0, y, bar(V_FULL + slot));
-                    tma_load_2d(dst + kHalfBytes, &tm_v, 64, y, bar(V_FULL + slot));
-                }
+                if (lane < n_pages)
+                    tma_load_page(sbase + kOffV + slot * kOperandBytes + lane * 4096, &tm_v, page_head, bar(V_FULL + slot), stream_once);
             }
             g = seg.tile_begin + t_last;
         }
@@ -189,10 +193,9 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 tc_fence_after();
                 const uint32_t qa = sbase + kOffQ, ka = sbase + kOffK + slot * kOperandBytes;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                    umma_bf16(tmem_s[sb], smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), idesc_qk, ks > 0);
-                }
+                for (int ks = 0; ks < 8; ++ks)               // Q: two 64-dim blocks of 128 rows; K: dim halves 1 KiB apart inside a page
+                    umma_bf16(tmem_s[sb], smem_desc(qa + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024),
+                              smem_desc(ka + (ks >> 2) * 1024 + (ks & 3) * 32, 16, 2048), idesc_qk, ks > 0);
                 umma_commit(bar(K_EMPTY + slot));
                 umma_commit(bar(S_FULL + sb));
                 return true;
@@ -215,8 +218,8 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint32_t aoff = (ks >> 2) * kHalfBytes + (ks & 3) * 32;      // P: K-major over tokens
-                        const uint32_t boff = ks * 2048;                                    // V: 16 token rows per step
-                        umma_bf16(tmem_o, smem_desc(pa + aoff, 16, 1024), smem_desc(va + boff, kHalfBytes, 1024), idesc_pv,
+                        const uint32_t boff = ks * 4096;                                    // V: one page (16 tokens) per step
+                        umma_bf16(tmem_o, smem_desc(pa + aoff, 16, 1024), smem_desc(va + boff, 1024, 2048), idesc_pv,
                                   (j > 0 || ks > 0) ? 1u : 0u);
                     }
                     umma_commit(bar(V_EMPTY + slot));
@@ -261,7 +264,7 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 }
             }
             fence_proxy_async();
-            mbar_arrive(bar(Q_FULL));
+            warp_arrive(bar(Q_FULL), lane);
 
             float m_ref = -INFINITY, l_sum = 0.f;           // reference max (log2 units); sum over this thread's columns
             const int Ltok = seg.n_tokens;
@@ -281,7 +284,7 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 tmem_ld32(tmem_s[sb] + lane_base + (uint32_t)col0 + 32u, reinterpret_cast<uint32_t*>(sv) + 32);
                 tmem_wait_ld();
                 tc_fence_before();
-                mbar_arrive(bar(S_FREE + sb));               // the scores are in registers: S may be overwritten
+                warp_arrive(bar(S_FREE + sb), lane);         // the scores are in registers: S may be overwritten
                 if (need_mask) {
 #pragma unroll
                     for (int c = 0; c < W; ++c) {
@@ -290,9 +293,10 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                         if (!ok) sv[c] = -INFINITY;
                     }
                 }
-                float mx = -INFINITY;
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};     // four independent chains
 #pragma unroll
-                for (int c = 0; c < W; ++c) mx = fmaxf(mx, sv[c]);
+                for (int c = 0; c < W; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], sv[c]);
+                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 // the row maximum over both halves
                 float* x = xch + (it & 1) * 2 * kRows;
                 x[half * kRows + L] = mx;
@@ -324,13 +328,14 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
 
                 // probabilities -> this thread's half of its row of P (bf16) in shared memory
                 const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+                float l4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int q8 = 0; q8 < W / 8; ++q8) {
                     float pr[8];
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         pr[c] = ex2(fmaf(sv[8 * q8 + c], p.scale_log2, neg_m));       // masked: ex2(-inf) = 0
-                        l_sum += pr[c];
+                        l4[c & 3] += pr[c];
                     }
                     uint4 pk;
                     __nv_bfloat162 h0 = __floats2bfloat162_rn(pr[0], pr[1]), h1 = __floats2bfloat162_rn(pr[2], pr[3]);
@@ -339,6 +344,7 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                     pk.z = *reinterpret_cast<uint32_t*>(&h2); pk.w = *reinterpret_cast<uint32_t*>(&h3);
                     *reinterpret_cast<uint4*>(smem + kOffP + kmajor_chunk_off(L, (col0 >> 3) + q8)) = pk;
                 }
+                l_sum += (l4[0] + l4[1]) + (l4[2] + l4[3]);
 
                 // last tile of a private segment: zero the V rows of the loaded pages past the branch end
                 if (need_mask) {
@@ -350,13 +356,14 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                         if (!alive) break;
                         for (int idx = tid; idx < (n_loaded - n_valid) * 16; idx += kSoftmaxThreads) {
                             const int row = n_valid + idx / 16, c = idx % 16;
-                            *reinterpret_cast<uint4*>(smem + kOffV + slot * kOperandBytes + (c >> 3) * kHalfBytes + row * 128 + ((c & 7) << 4)) =
-                                make_uint4(0, 0, 0, 0);
+                            // token `row` of the staged tile: page, token half, 8-token group row; both dim halves
+                            *reinterpret_cast<uint4*>(smem + kOffV + slot * kOperandBytes + (row >> 4) * 4096 + ((row >> 3) & 1) * 2048 +
+                                                      (c >> 3) * 1024 + (row & 7) * 128 + ((c & 7) << 4)) = make_uint4(0, 0, 0, 0);
                         }
                     }
                 }
                 fence_proxy_async();
-                mbar_arrive(bar(P_FULL));
+                warp_arrive(bar(P_FULL), lane);
             }
             if (!alive) break;
 
@@ -467,10 +474,10 @@ int umma_copies(int nr) { (void)nr; return 1; }
 cudaError_t launch_attn_umma(Ctx* c, const AttnParams& p, cudaStream_t st) {
     if (p.N > kUmmaMaxBranches) return cudaErrorInvalidValue;
     cudaError_t err = cudaSuccess;
-    const CUtensorMap* mk = umma_pool_map(c, p.k_pages, 0, &err);
+    const CUtensorMap* mk = umma_pool_map(c, p.k_pages, 1, &err);
     if (!mk) return err;
     const CUtensorMap mk_copy = *mk;                       // the cache may reallocate on the next insert
-    const CUtensorMap* mv = umma_pool_map(c, p.v_pages, 0, &err);
+    const CUtensorMap* mv = umma_pool_map(c, p.v_pages, 1, &err);
     if (!mv) return err;
     static bool attr_set[64] = {};                          // the attribute is per device
     if (c->device < 0 || c->device >= 64 || !attr_set[c->device]) {
