@@ -49,8 +49,7 @@ constexpr uint32_t kTmemCols = 512;
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int kOffQ = 0;
-constexpr int kOffP = kOffQ + kOperandBytes;
-constexpr int kOffK = kOffP + kOperandBytes;
+constexpr int kOffK = kOffQ + kOperandBytes;
 constexpr int kOffV = kOffK + kRing * kOperandBytes;
 constexpr int kOffBar = kOffV + kRing * kOperandBytes;        // 196608
 constexpr int kNumBars = 16;
@@ -100,17 +99,15 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
     const int g_end = min(total, g_begin + tpc);
     if (g_begin >= g_end) return;                          // uniform: nothing to do for this CTA
 
-    // ---- set-up: zero P and the V ring (nothing non-finite may ever meet a zero weight), barriers, TMEM ----
-    for (int i = tid; i < (kOperandBytes + kRing * kOperandBytes) / 16; i += kThreadsUmma) {
-        const int off = i * 16 < kOperandBytes ? kOffP + i * 16 : kOffV + (i * 16 - kOperandBytes);
-        *reinterpret_cast<uint4*>(smem + off) = make_uint4(0, 0, 0, 0);
-    }
+    // ---- set-up: zero the V ring (nothing non-finite may ever meet a zero weight), barriers, TMEM ----
+    for (int i = tid; i < kRing * kOperandBytes / 16; i += kThreadsUmma)
+        *reinterpret_cast<uint4*>(smem + kOffV + i * 16) = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
         misc[0] = 0;
         for (int i = 0; i < kRing; ++i) {
             mbar_init(bar(K_FULL + i), 1); mbar_init(bar(K_EMPTY + i), 1);
             mbar_init(bar(V_FULL + i), 1); mbar_init(bar(V_EMPTY + i), 1);
-            mbar_init(bar(S_FULL + i), 1); mbar_init(bar(S_FREE + i), kSoftmaxThreads / 32);
+            mbar_init(bar(S_FULL + i), 1);
         }
         mbar_init(bar(P_FULL), kSoftmaxThreads / 32); mbar_init(bar(PV_DONE), 1); mbar_init(bar(Q_FULL), kSoftmaxThreads / 32);   // the softmax warps arrive once per warp
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -189,7 +186,8 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
             auto issue_qk = [&](int j) -> bool {
                 const int slot = j % kRing, sb = j & 1;
                 if (!mbar_wait(bar(K_FULL + slot), (j / kRing) & 1, ab)) return false;
-                if (!mbar_wait(bar(S_FREE + sb), ((j >> 1) & 1) ^ 1, ab)) return false;
+                // S buffer sb last held the probabilities of tile j - 2, read by that tile's second contraction,
+                // which was issued before this one: the tensor pipe keeps the order
                 tc_fence_after();
                 const uint32_t qa = sbase + kOffQ, ka = sbase + kOffK + slot * kOperandBytes;
 #pragma unroll
@@ -214,13 +212,14 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                     alive = mbar_wait(bar(P_FULL), cur & 1, ab) && mbar_wait(bar(V_FULL + slot), (cur / kRing) & 1, ab);
                     if (!alive) break;
                     tc_fence_after();
-                    const uint32_t pa = sbase + kOffP, va = sbase + kOffV + slot * kOperandBytes;
+                    const uint32_t va = sbase + kOffV + slot * kOperandBytes;
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t aoff = (ks >> 2) * kHalfBytes + (ks & 3) * 32;      // P: K-major over tokens
+                        // P: the A operand straight from TMEM, 16 tokens = 8 columns of packed bf16 pairs per step; the
+                        // two halves of a row sit at columns 0 and 64 of the tile's score buffer (see the softmax warps)
+                        const uint32_t pa = tmem_s[cur & 1] + (uint32_t)((ks >> 2) * 64 + (ks & 3) * 8);
                         const uint32_t boff = ks * 4096;                                    // V: one page (16 tokens) per step
-                        umma_bf16(tmem_o, smem_desc(pa + aoff, 16, 1024), smem_desc(va + boff, 1024, 2048), idesc_pv,
-                                  (j > 0 || ks > 0) ? 1u : 0u);
+                        umma_bf16_tmem_a(tmem_o, pa, smem_desc(va + boff, 1024, 2048), idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
                     }
                     umma_commit(bar(V_EMPTY + slot));
                     umma_commit(bar(PV_DONE));
@@ -283,8 +282,6 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 tmem_ld32(tmem_s[sb] + lane_base + (uint32_t)col0, reinterpret_cast<uint32_t*>(sv));
                 tmem_ld32(tmem_s[sb] + lane_base + (uint32_t)col0 + 32u, reinterpret_cast<uint32_t*>(sv) + 32);
                 tmem_wait_ld();
-                tc_fence_before();
-                warp_arrive(bar(S_FREE + sb), lane);         // the scores are in registers: S may be overwritten
                 if (need_mask) {
 #pragma unroll
                     for (int c = 0; c < W; ++c) {
@@ -326,25 +323,23 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 l_sum *= factor;
                 m_ref = m_new;
 
-                // probabilities -> this thread's half of its row of P (bf16) in shared memory
+                // probabilities -> bf16 pairs, written over the first 32 of this thread's own 64 score columns: the
+                // second contraction takes P from TMEM as its A operand (row = lane, two tokens per 32-bit column)
                 const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
                 float l4[4] = {0.f, 0.f, 0.f, 0.f};
+                uint32_t pw[W / 2];
 #pragma unroll
-                for (int q8 = 0; q8 < W / 8; ++q8) {
-                    float pr[8];
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        pr[c] = ex2(fmaf(sv[8 * q8 + c], p.scale_log2, neg_m));       // masked: ex2(-inf) = 0
-                        l4[c & 3] += pr[c];
-                    }
-                    uint4 pk;
-                    __nv_bfloat162 h0 = __floats2bfloat162_rn(pr[0], pr[1]), h1 = __floats2bfloat162_rn(pr[2], pr[3]);
-                    __nv_bfloat162 h2 = __floats2bfloat162_rn(pr[4], pr[5]), h3 = __floats2bfloat162_rn(pr[6], pr[7]);
-                    pk.x = *reinterpret_cast<uint32_t*>(&h0); pk.y = *reinterpret_cast<uint32_t*>(&h1);
-                    pk.z = *reinterpret_cast<uint32_t*>(&h2); pk.w = *reinterpret_cast<uint32_t*>(&h3);
-                    *reinterpret_cast<uint4*>(smem + kOffP + kmajor_chunk_off(L, (col0 >> 3) + q8)) = pk;
+                for (int c = 0; c < W; c += 2) {
+                    const float e0 = ex2(fmaf(sv[c], p.scale_log2, neg_m));            // masked: ex2(-inf) = 0
+                    const float e1 = ex2(fmaf(sv[c + 1], p.scale_log2, neg_m));
+                    l4[(c >> 1) & 1] += e0; l4[2 + ((c >> 1) & 1)] += e1;
+                    const __nv_bfloat162 h = __floats2bfloat162_rn(e0, e1);          // the even token in the low half
+                    pw[c >> 1] = *reinterpret_cast<const uint32_t*>(&h);
                 }
                 l_sum += (l4[0] + l4[1]) + (l4[2] + l4[3]);
+                tmem_st32(tmem_s[sb] + lane_base + (uint32_t)col0, pw);
+                tmem_wait_st();
+                tc_fence_before();
 
                 // last tile of a private segment: zero the V rows of the loaded pages past the branch end
                 if (need_mask) {
