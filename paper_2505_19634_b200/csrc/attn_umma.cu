@@ -5,18 +5,22 @@
 // 128 KV tokens of one KV head = 8 pages gathered through the block table, each page-head tile
 // (16 tokens x 128 dims, 4 KiB contiguous) arriving as one 128-byte-swizzled 5-D TMA box.
 //
-//   warp 8      producer: per tile, arms the K and V "full" barriers with the byte count and
-//               issues the TMA boxes (K ring and V ring, 2 slots x 32 KiB each)
-//   warp 9      MMA issuer (one thread): S = Q K^T into one of two TMEM buffers, then
+//   warps 8, 9  producers, one for the K tiles (ring of 3 slots x 32 KiB) and one for the V tiles (ring
+//               of 2): per tile the warp arms the slot's "full" barrier with the byte count and issues
+//               one TMA box per page.  K tiles are wanted a whole softmax step before their V tiles.
+//   warp 10     MMA issuer (one thread): S = Q K^T into one of two TMEM buffers, then
 //               O (+)= P V once the softmax warps have published P; frees ring slots with
 //               tcgen05.commit
 //   warps 0-7   softmax: two threads per query row (TMEM lane), each on one half of the tile's 128 key
 //               columns.  A thread reads its 64 scores once, the pair agrees on the row maximum
-//               through shared memory, and each writes its half of the row of P (bf16, swizzled
-//               K-major) for the second contraction.  O is rescaled in TMEM only when the max moved
-//               by more than 2^8 (the final result is exact either way, l carries the same
-//               reference); each thread keeps the sum of its own columns; the piece's partial
-//               (m, l, O) is written at the end.
+//               through shared memory, and each writes its probabilities as packed bf16 pairs over
+//               the first half of its own score columns: the second contraction takes P from TMEM as
+//               its A operand, so there is no P buffer in shared memory and a tile's exponentials
+//               do not wait for the previous tile's second contraction.  O is rescaled in TMEM only
+//               when the max moved by more than 2^8 (the final result is exact either way, l carries
+//               the same reference; only then does a warp wait for the previous contraction); each
+//               thread keeps the sum of its own columns; the piece's partial (m, l, O) is written at
+//               the end.
 //
 // This is the kernel for many query rows per KV head (draft trees: nodes x GQA group rows); with few rows
 // most of the 128-row tile is padding and the token-major kernel (attn_umma_t.cu) is the one to use.
@@ -40,18 +44,18 @@ using namespace ptx;
 constexpr int kTile = kUmmaTileTokens;            // 128 tokens
 constexpr int kRows = kUmmaRows;                   // 128 = MMA M
 constexpr int kSoftmaxThreads = 256;                 // 8 warps: (TMEM lane quarter, column half)
-constexpr int kThreadsUmma = kSoftmaxThreads + 64;
-constexpr int kProducerWarp = kSoftmaxThreads / 32, kMmaWarp = kProducerWarp + 1;
+constexpr int kThreadsUmma = kSoftmaxThreads + 96;
+constexpr int kProducerWarp = kSoftmaxThreads / 32, kMmaWarp = kProducerWarp + 2;   // producers: K, then V
 constexpr int kHalfBytes = kRows * 128;            // one 64-element K-block of a 128-row operand: 16 KiB
 constexpr int kOperandBytes = 2 * kHalfBytes;      // 32 KiB
-constexpr int kRing = 2;
+constexpr int kRingK = 3, kRingV = 2;                 // K tiles are wanted a whole softmax step before their V tiles
 constexpr uint32_t kTmemCols = 512;
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int kOffQ = 0;
 constexpr int kOffK = kOffQ + kOperandBytes;
-constexpr int kOffV = kOffK + kRing * kOperandBytes;
-constexpr int kOffBar = kOffV + kRing * kOperandBytes;        // 196608
+constexpr int kOffV = kOffK + kRingK * kOperandBytes;
+constexpr int kOffBar = kOffV + kRingV * kOperandBytes;
 constexpr int kNumBars = 16;
 constexpr int kOffMisc = kOffBar + kNumBars * 8;
 constexpr int kOffXch = kOffMisc + 64;                         // float[5][128]: row maxima of two tiles x two halves, row sums
@@ -59,7 +63,10 @@ constexpr int kOffCum = kOffXch + 5 * kRows * 4;
 constexpr int kUmmaMaxBranches = 1024;
 constexpr int kSmemBytes = kOffCum + (kUmmaMaxBranches + 1) * 4 + 1024;   // + slack for manual alignment
 
-enum Bar { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, S_FULL = 8, S_FREE = 10, P_FULL = 12, PV_DONE = 13, Q_FULL = 14 };
+// PV_DONE: two barriers, tile j completes PV_DONE + (j & 1), so that a waiter's parity follows from the tile index alone
+// even when it has not waited for every tile
+enum Bar { K_FULL = 0, K_EMPTY = 3, V_FULL = 6, V_EMPTY = 8, S_FULL = 10, PV_DONE = 12, P_FULL = 14, Q_FULL = 15 };
+static_assert(kRingK == 3 && kRingV == 2 && kNumBars == 16, "barrier numbering");
 
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128; B either K-major or MN-major.
 __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) { return ptx::instr_desc(128, 128, false, b_mn_major); }
@@ -100,16 +107,16 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
     if (g_begin >= g_end) return;                          // uniform: nothing to do for this CTA
 
     // ---- set-up: zero the V ring (nothing non-finite may ever meet a zero weight), barriers, TMEM ----
-    for (int i = tid; i < kRing * kOperandBytes / 16; i += kThreadsUmma)
+    for (int i = tid; i < kRingV * kOperandBytes / 16; i += kThreadsUmma)
         *reinterpret_cast<uint4*>(smem + kOffV + i * 16) = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
         misc[0] = 0;
-        for (int i = 0; i < kRing; ++i) {
-            mbar_init(bar(K_FULL + i), 1); mbar_init(bar(K_EMPTY + i), 1);
+        for (int i = 0; i < kRingK; ++i) { mbar_init(bar(K_FULL + i), 1); mbar_init(bar(K_EMPTY + i), 1); }
+        for (int i = 0; i < 2; ++i) {
             mbar_init(bar(V_FULL + i), 1); mbar_init(bar(V_EMPTY + i), 1);
             mbar_init(bar(S_FULL + i), 1);
         }
-        mbar_init(bar(P_FULL), kSoftmaxThreads / 32); mbar_init(bar(PV_DONE), 1); mbar_init(bar(Q_FULL), kSoftmaxThreads / 32);   // the softmax warps arrive once per warp
+        mbar_init(bar(P_FULL), kSoftmaxThreads / 32); mbar_init(bar(PV_DONE), 1); mbar_init(bar(PV_DONE + 1), 1); mbar_init(bar(Q_FULL), kSoftmaxThreads / 32);   // the softmax warps arrive once per warp
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMmaWarp) {
@@ -124,9 +131,15 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
     const uint32_t tmem_s[2] = {tmem, tmem + 128u};
     const uint32_t tmem_o = tmem + 256u;
 
-    if (warp == kProducerWarp) {
-        // =========================== producer ===========================
-        int it = 0;                                         // tiles issued by this CTA
+    if (warp == kProducerWarp || warp == kProducerWarp + 1) {
+        // =========================== producers: one warp for the K tiles, one for the V tiles ===========================
+        const int op = warp - kProducerWarp;               // 0: K, 1: V
+        const int ring_n = op == 0 ? kRingK : kRingV;
+        const int full0 = op == 0 ? K_FULL : V_FULL, empty0 = op == 0 ? K_EMPTY : V_EMPTY;
+        const uint32_t ring_base = sbase + (op == 0 ? kOffK : kOffV);
+        const CUtensorMap* tm = op == 0 ? &tm_k : &tm_v;
+        int it = 0;                                         // tiles issued by this warp
+        int slot = 0, round = 0;                            // it % ring_n, (it / ring_n) & 1
         int g = g_begin;
         bool alive = true;
         const uint64_t stream_once = l2_policy_evict_first();
@@ -135,8 +148,6 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
             const int t_first = g - seg.tile_begin, t_last = min(seg.n_tiles, g_end - seg.tile_begin);
             const int32_t* bt = p.block_table + (size_t)(seg.kind == 0 ? 0 : seg.b) * p.max_blocks;
             for (int t = t_first; t < t_last && alive; ++t, ++it) {
-                const int slot = it % kRing;
-                const uint32_t par = ((it / kRing) & 1) ^ 1;
                 const int tok0 = t * kTile;
                 const int n_pages = ceil_div(min(kTile, seg.n_tokens - tok0), kPage);
                 int page = 0;
@@ -144,36 +155,26 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 // one box per page-head tile (4 KiB), laid out [token half][dim half][8 tokens][128 bytes], so the
                 // pages of a tile form one MMA operand with 2 KiB between its 8-token groups
                 const int page_head = page * p.Hkv + seg.kvh;
-                // K
                 if (lane == 0) {
-                    alive = mbar_wait(bar(K_EMPTY + slot), par, ab);
-                    if (alive) mbar_arrive_expect_tx(bar(K_FULL + slot), (uint32_t)n_pages * 4096u);
+                    alive = mbar_wait(bar(empty0 + slot), round ^ 1, ab);
+                    if (alive) mbar_arrive_expect_tx(bar(full0 + slot), (uint32_t)n_pages * 4096u);
                 }
                 alive = __shfl_sync(0xffffffffu, alive, 0);
                 if (!alive) break;
                 if (lane < n_pages)
-                    tma_load_page(sbase + kOffK + slot * kOperandBytes + lane * 4096, &tm_k, page_head, bar(K_FULL + slot), stream_once);
-                // V
-                if (lane == 0) {
-                    alive = mbar_wait(bar(V_EMPTY + slot), par, ab);
-                    if (alive) mbar_arrive_expect_tx(bar(V_FULL + slot), (uint32_t)n_pages * 4096u);
-                }
-                alive = __shfl_sync(0xffffffffu, alive, 0);
-                if (!alive) break;
-                if (lane < n_pages)
-                    tma_load_page(sbase + kOffV + slot * kOperandBytes + lane * 4096, &tm_v, page_head, bar(V_FULL + slot), stream_once);
+                    tma_load_page(ring_base + slot * kOperandBytes + lane * 4096, tm, page_head, bar(full0 + slot), stream_once);
+                if (++slot == ring_n) { slot = 0; round ^= 1; }
             }
             g = seg.tile_begin + t_last;
         }
         // Copies this warp started must have landed before the CTA may exit: the consumers wait on
         // the same phases in the normal case; after an abort wait for them here (bounded).
         if (*ab.flag && lane == 0) {
-            for (int back = 1; back <= kRing && back <= it; ++back) {
+            for (int back = 1; back <= ring_n && back <= it; ++back) {
                 const int j = it - back;
-                const Abort quiet{misc + 2, p.status};       // do not re-raise; misc[2] is scratch
-                misc[2] = 0;
-                mbar_wait(bar(K_FULL + j % kRing), (j / kRing) & 1, quiet);
-                mbar_wait(bar(V_FULL + j % kRing), (j / kRing) & 1, quiet);
+                const Abort quiet{misc + 2 + op, p.status};  // do not re-raise; misc[2], misc[3] are scratch
+                misc[2 + op] = 0;
+                mbar_wait(bar(full0 + j % ring_n), (j / ring_n) & 1, quiet);
             }
         }
     } else if (warp == kMmaWarp) {
@@ -184,8 +185,8 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
             int g = g_begin;
             bool alive = true;
             auto issue_qk = [&](int j) -> bool {
-                const int slot = j % kRing, sb = j & 1;
-                if (!mbar_wait(bar(K_FULL + slot), (j / kRing) & 1, ab)) return false;
+                const int slot = j % kRingK, sb = j & 1;
+                if (!mbar_wait(bar(K_FULL + slot), (j / kRingK) & 1, ab)) return false;
                 // S buffer sb last held the probabilities of tile j - 2, read by that tile's second contraction,
                 // which was issued before this one: the tensor pipe keeps the order
                 tc_fence_after();
@@ -208,8 +209,8 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 alive = issue_qk(it);
                 for (int j = 0; j < n && alive; ++j) {
                     if (j + 1 < n) { alive = issue_qk(it + j + 1); if (!alive) break; }
-                    const int cur = it + j, slot = cur % kRing;
-                    alive = mbar_wait(bar(P_FULL), cur & 1, ab) && mbar_wait(bar(V_FULL + slot), (cur / kRing) & 1, ab);
+                    const int cur = it + j, slot = cur % kRingV;
+                    alive = mbar_wait(bar(P_FULL), cur & 1, ab) && mbar_wait(bar(V_FULL + slot), (cur / kRingV) & 1, ab);
                     if (!alive) break;
                     tc_fence_after();
                     const uint32_t va = sbase + kOffV + slot * kOperandBytes;
@@ -222,7 +223,7 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                         umma_bf16_tmem_a(tmem_o, pa, smem_desc(va + boff, 1024, 2048), idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
                     }
                     umma_commit(bar(V_EMPTY + slot));
-                    umma_commit(bar(PV_DONE));
+                    umma_commit(bar(PV_DONE + (cur & 1)));
                 }
                 it += n; ++piece;
                 g = seg.tile_begin + t_last;
@@ -303,13 +304,11 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 const float m_new = move ? mx : m_ref;
                 const float factor = (move && m_ref != -INFINITY) ? ex2(m_ref - m_new) : 1.f;
 
-                // the previous tile's P.V must be finished before P is overwritten or O touched
-                if (it > 0) {
-                    alive = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE), (it - 1) & 1, ab));
+                if (t > t_first && __any_sync(0xffffffffu, factor != 1.f)) {     // this thread's half of its O row
+                    // O is touched: the previous tile's second contraction must have finished
+                    alive = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, ab));
                     if (!alive) break;
                     tc_fence_after();
-                }
-                if (t > t_first && __any_sync(0xffffffffu, factor != 1.f)) {     // this thread's half of its O row
                     for (int ch = 0; ch < 2; ++ch) {
                         uint32_t ov[32];
                         tmem_ld32(tmem_o + lane_base + (uint32_t)(col0 + 32 * ch), ov);
@@ -346,8 +345,8 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                     const int n_valid = min(kTile, Ltok - tok0);
                     const int n_loaded = ceil_div(n_valid, kPage) * kPage;
                     if (n_valid < n_loaded) {
-                        const int slot = it % kRing;
-                        alive = __all_sync(0xffffffffu, mbar_wait(bar(V_FULL + slot), (it / kRing) & 1, ab));
+                        const int slot = it % kRingV;
+                        alive = __all_sync(0xffffffffu, mbar_wait(bar(V_FULL + slot), (it / kRingV) & 1, ab));
                         if (!alive) break;
                         for (int idx = tid; idx < (n_loaded - n_valid) * 16; idx += kSoftmaxThreads) {
                             const int row = n_valid + idx / 16, c = idx % 16;
@@ -363,7 +362,7 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
             if (!alive) break;
 
             // ---- piece epilogue: partial (m, l, O) ----
-            alive = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE), (it - 1) & 1, ab));
+            alive = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, ab));
             if (!alive) break;
             tc_fence_after();
             float* po; float2* pml;
