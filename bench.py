@@ -437,8 +437,30 @@ def run_ours(args, shape):
         h2d = (q_host.numel() * 2 + h_bt.numel() * 4 + h_lens.numel() * 4 + h_p.numel() * 4 + h_q.numel() * 4 +
                h_t.numel() * 4 + h_u.numel() * 4)
         d2h = out_host.numel() * 2 + 8 * N
+        # the same step with the accept pass fed with bf16 logits (half the bytes of the two distribution tensors)
+        e2e_logits = None
+        if world == 1:
+            import paper_2505_19634_b200 as tts
+            lc = ti.make_accept_logits_case(N, g, V, shape.logit_sigma, seed + 3, bf16=True)
+            h_tl, h_dl = pin(lc.target_logits.view(np.int16)), pin(lc.draft_logits.view(np.int16))
+            h_lt, h_lu = pin(lc.draft_tokens), pin(lc.uniforms)
+
+            def step_host_logits():
+                ctx.tts_verify_step_host_logits(L, q_host, ds.k_pools, ds.v_pools, h_bt, shape.prefix_len, h_lens, N, g,
+                                                h_tl, h_dl, tts.LOGITS_BF16, h_lt, h_lu, V, out_host, h_al, h_nt)
+            for _ in range(2):
+                step_host_logits()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(e2e_steps):
+                step_host_logits()
+            torch.cuda.synchronize()
+            lms = (time.perf_counter() - t0) / e2e_steps * 1e3
+            e2e_logits = {"ms_per_step": lms, "value": step_bytes / (lms * 1e-3) / 1e9, "unit": "GB/s",
+                          "h2d_bytes_per_step": h2d - (h_p.numel() + h_q.numel()) * 4 + (h_tl.numel() + h_dl.numel()) * 2,
+                          "d2h_bytes_per_step": d2h, "call": "tts_verify_step_host_logits, bf16 logits"}
     else:
-        e2e_ms, h2d, d2h = 0.0, 0, 0
+        e2e_ms, h2d, d2h, e2e_logits = 0.0, 0, 0, None
 
     ms, e2e_ms, launches = aggregate_over_ranks(ms, e2e_ms, launches, world, dev)
 
@@ -486,7 +508,8 @@ def run_ours(args, shape):
                        "attn_impl": "auto"},
             "clocks": clocks,
             "e2e": {"value": total_bytes / (e2e_ms * 1e-3) / 1e9 if e2e_ms else None, "unit": "GB/s", "ms_per_step": e2e_ms,
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "call": "tts_verify_step_host, fp32 probabilities"},
+            "e2e_logits": e2e_logits,
             "gpu_launches": launches,
             "roofline": roof,
             "cpu_baseline": {"value": cb_bytes / cb_s / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
