@@ -143,8 +143,9 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
         int g = g_begin;
         bool alive = true;
         const uint64_t stream_once = l2_policy_evict_first();
-        while (g < g_end && alive) {
-            const SegInfo seg = segment_of_tile(p, cum, g);
+        SegInfo seg = segment_of_tile(p, cum, g);           // the first piece by search, the following ones by stepping
+        for (bool first_piece = true; g < g_end && alive; first_piece = false) {
+            if (!first_piece) seg = next_segment(p, cum, seg);
             const int t_first = g - seg.tile_begin, t_last = min(seg.n_tiles, g_end - seg.tile_begin);
             const int32_t* bt = p.block_table + (size_t)(seg.kind == 0 ? 0 : seg.b) * p.max_blocks;
             for (int t = t_first; t < t_last && alive; ++t, ++it) {
@@ -199,8 +200,9 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
                 umma_commit(bar(S_FULL + sb));
                 return true;
             };
-            while (g < g_end && alive) {
-                const SegInfo seg = segment_of_tile(p, cum, g);
+            SegInfo seg = segment_of_tile(p, cum, g);
+            for (bool first_piece = true; g < g_end && alive; first_piece = false) {
+                if (!first_piece) seg = next_segment(p, cum, seg);
                 const int t_first = g - seg.tile_begin, t_last = min(seg.n_tiles, g_end - seg.tile_begin);
                 const int n = t_last - t_first;
                 alive = mbar_wait(bar(Q_FULL), piece & 1, ab);
@@ -240,8 +242,9 @@ attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, c
         int it = 0;
         int g = g_begin;
         bool alive = true;
-        while (g < g_end && alive) {
-            const SegInfo seg = segment_of_tile(p, cum, g);
+        SegInfo seg = segment_of_tile(p, cum, g);
+        for (bool first_piece = true; g < g_end && alive; first_piece = false) {
+            if (!first_piece) seg = next_segment(p, cum, seg);
             const int t_first = g - seg.tile_begin, t_last = min(seg.n_tiles, g_end - seg.tile_begin);
             const bool valid = L < seg.n_rows;
 
