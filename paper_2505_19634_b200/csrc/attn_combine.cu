@@ -127,7 +127,6 @@ __global__ void __launch_bounds__(512) attn_combine_groups_kernel(const AttnPara
 
 cudaError_t launch_attn_combine(const AttnParams& main_params, cudaStream_t st) {
     AttnParams p = main_params;
-    p.lens_smem = 0;                     // this kernel's shared memory holds the tile prefix only (N + 1 ints)
     if (p.copies == 1 && p.copies_pre == 1 && p.n_rb_priv <= kMaxPrivBlocks && p.nr <= 2 * p.rb_rows) {
         const int threads = min(512, (p.nr * 16 + 31) / 32 * 32);        // 128 registers each: a row's loads are all in flight at once
         attn_combine_groups_kernel<<<p.N * p.Hkv, threads, (p.N + 1) * sizeof(int), st>>>(p);

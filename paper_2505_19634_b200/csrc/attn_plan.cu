@@ -31,7 +31,6 @@ __device__ AttnParams set_params(const AttnParams& p, const PrefixSets& sets, in
     q.n_rb_pre = ceil_div(q.N * p.nr, p.rb_rows);
     q.n_pre = q.P > 0 ? p.Hkv * q.n_rb_pre : 0;
     q.tiles_pre = ceil_div(q.P, p.tile_tokens);
-    q.lens_smem = 0;
     return q;
 }
 
@@ -163,7 +162,6 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(const AttnParam
 
 cudaError_t launch_attn_plan(const AttnParams& main_params, const PrefixSets& sets, cudaStream_t st) {
     AttnParams p = main_params;
-    p.lens_smem = 0;
     const size_t smem = (size_t)(p.N + sets.n_sets + 2 * sets.n_sets + 1 + p.grid + 1) * sizeof(int) +
                         (size_t)p.grid * 2 * sizeof(FirstTile);
     attn_plan_kernel<<<1, kPlanThreads, smem, st>>>(p, sets, const_cast<CtaPlan*>(p.plan_cta),

@@ -70,7 +70,6 @@ struct AttnParams {
     int tile_tokens;
     int grid;                       // CTAs of the main kernel
     int out_dtype, debug;
-    int lens_smem;                  // the kernel keeps the branch lengths behind cum[] in shared memory (2N + 1 ints)
     float scale_log2;               // softmax scale * log2(e)
 };
 
@@ -89,12 +88,10 @@ struct SegInfo {
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 // cum[b] = tiles of branches < b (per private segment of that branch), cum[N] = sum.
-// Must be called by all threads of the block; cum lives in shared memory (N+1 ints, followed by
-// the N branch lengths themselves when p.lens_smem is set: the schedule then needs no global load).
+// Must be called by all threads of the block; cum lives in shared memory (N+1 ints).
 __device__ inline void build_branch_tile_prefix(const AttnParams& p, int* cum) {
     for (int b = threadIdx.x; b < p.N; b += blockDim.x) {
         int L = p.branch_lens[b];
-        if (p.lens_smem) cum[p.N + 1 + b] = L;
         L = L < 0 ? 0 : L;
         cum[b + 1] = ceil_div(L, p.tile_tokens);
     }
@@ -118,7 +115,8 @@ __device__ inline void build_branch_tile_prefix(const AttnParams& p, int* cum) {
 }
 
 __device__ __forceinline__ int branch_len(const AttnParams& p, const int* cum, int b) {
-    return p.lens_smem ? cum[p.N + 1 + b] : p.branch_lens[b];
+    (void)cum;
+    return p.branch_lens[b];
 }
 
 // a / b and a % b for 0 <= a < 2^31 with a quotient below 2^22, 0 < b: float estimate, corrected
@@ -189,23 +187,6 @@ __device__ inline SegInfo segment_of_tile(const AttnParams& p, const int* cum, i
         if (group_tile_begin(p, cum, mid) <= g) lo = mid; else hi = mid - 1;
     }
     return segment_in_group(p, cum, lo, g);
-}
-
-// The search alone (the group of tile g) for a value of g that is uniform over the thread block,
-// called by all its threads: the candidates of a round are tested by one thread each, so the search
-// takes one round per factor of blockDim.x in the number of groups instead of one dependent step
-// per factor of two.
-__device__ inline int group_of_tile_block(const AttnParams& p, const int* cum, int g) {
-    int lo = 0, n = p.N * p.Hkv;               // the group is in [lo, lo + n); group lo begins at or before g
-    while (n > 1) {
-        const int stride = ceil_div(n, (int)blockDim.x);
-        const int idx = lo + (int)threadIdx.x * stride;
-        const int c = __syncthreads_count(idx < lo + n && group_tile_begin(p, cum, idx) <= g);   // >= 1: thread 0
-        const int end = lo + n;
-        lo += (c - 1) * stride;
-        n = min(stride, end - lo);
-    }
-    return lo;
 }
 
 // The segment after s in the tile list (the caller knows there is one): the next row block of the
