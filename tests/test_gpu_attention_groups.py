@@ -110,3 +110,15 @@ def test_group_argument_errors():
             ctx.tts_verify_attn_groups(z, z, z, z, sizes, pre, z, 6, c.gamma, z)
         assert ei.value.status == -1
     ctx.close()
+
+
+def test_groups_under_a_capped_grid():
+    """The cut of the concatenated tile lists moves with the number of CTAs; the result must not."""
+    c = ti.make_group_case(seed=45, **CASES["ragged_groups"])
+    ti.poison_unused_slots_groups(c)
+    want = oracle_groups(c)
+    for cap in (1, 3, 29):
+        ctx = tts.TtsContext(c.n_q_heads, c.n_kv_heads, c.n_branches, c.gamma + 1, c.max_blocks, c.num_pages,
+                             attn_impl=tts.ATTN_TCGEN05_TOKEN_MAJOR, debug_bounds=True, max_ctas=cap)
+        assert_attn_close(run_groups(c, tts.ATTN_TCGEN05_TOKEN_MAJOR, ctx=ctx, planned=True), want, what=f"cap {cap}")
+        ctx.close()

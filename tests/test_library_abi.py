@@ -153,3 +153,23 @@ def test_create_rejects_bad_configs_without_a_gpu():
         assert lib.tts_create(ctypes.byref(cfg), ctypes.byref(h)) == want, bad
         assert not h.value
     assert lib.tts_create(None, ctypes.byref(h)) == -1
+
+
+def test_entry_points_reject_null_contexts_and_bad_groups_without_a_gpu():
+    """Host-side argument checks that need no device: every context-taking entry point returns
+    TTS_ERR_INVALID for a null context, and the group arrays of the multi-question calls are validated
+    before anything else."""
+    import ctypes
+    lib = tts.load_library()
+    i32 = lambda *v: (ctypes.c_int32 * len(v))(*v)
+    z = ctypes.c_void_p(0)
+    assert lib.tts_attn_plan(z, z, 16, z, 1, 1) == -1
+    assert lib.tts_attn_plan_drop(z) == -1
+    assert lib.tts_verify_attn(z, z, z, z, z, 16, z, 1, 0, 0, z) == -1
+    assert lib.tts_accept_logits(z, z, z, 0, z, z, 1, 0, 8, z, z) == -1
+    assert lib.tts_debug_wait_timeout(z, 1000000) == -1
+    assert lib.tts_kv_rollback(z, z, z, 1, 0) == -1
+    # groups: sizes must be >= 1 and add up to n_branches, at most 64 groups
+    for sizes, pre, n in (((2, 1), (16, 0), 4), ((2, 0, 2), (16, 0, 16), 4), ((1,) * 65, (0,) * 65, 65)):
+        assert lib.tts_verify_attn_groups(z, z, z, z, z, i32(*sizes), i32(*pre), len(sizes), z, n, 1, z) == -1
+        assert lib.tts_attn_plan_groups(z, z, i32(*sizes), i32(*pre), len(sizes), z, n, 2) == -1
