@@ -434,8 +434,11 @@ def run_ours(args, shape):
             step_host()
         torch.cuda.synchronize()
         e2e_ms = (time.perf_counter() - t0) / e2e_steps * 1e3
-        h2d = (q_host.numel() * 2 + h_bt.numel() * 4 + h_lens.numel() * 4 + h_p.numel() * 4 + h_q.numel() * 4 +
-               h_t.numel() * 4 + h_u.numel() * 4)
+        # the two probability tensors are pinned: the accept kernel reads its share of them in place over the host
+        # link (its algorithmic bytes), everything else is copied
+        h2d_copied = q_host.numel() * 2 + h_bt.numel() * 4 + h_lens.numel() * 4 + h_t.numel() * 4 + h_u.numel() * 4
+        h2d = h2d_copied + acc_bytes
+        h2d_all = h2d_copied + (h_p.numel() + h_q.numel()) * 4
         d2h = out_host.numel() * 2 + 8 * N
         # the same step with the accept pass fed with bf16 logits (half the bytes of the two distribution tensors)
         e2e_logits = None
@@ -457,10 +460,10 @@ def run_ours(args, shape):
             torch.cuda.synchronize()
             lms = (time.perf_counter() - t0) / e2e_steps * 1e3
             e2e_logits = {"ms_per_step": lms, "value": step_bytes / (lms * 1e-3) / 1e9, "unit": "GB/s",
-                          "h2d_bytes_per_step": h2d - (h_p.numel() + h_q.numel()) * 4 + (h_tl.numel() + h_dl.numel()) * 2,
+                          "h2d_bytes_per_step": h2d_copied + (h_tl.numel() + h_dl.numel()) * 2,
                           "d2h_bytes_per_step": d2h, "call": "tts_verify_step_host_logits, bf16 logits"}
     else:
-        e2e_ms, h2d, d2h, e2e_logits = 0.0, 0, 0, None
+        e2e_ms, h2d, d2h, e2e_logits, h_p, h_q = 0.0, 0, 0, None, None, None
 
     ms, e2e_ms, launches = aggregate_over_ranks(ms, e2e_ms, launches, world, dev)
 
@@ -508,7 +511,10 @@ def run_ours(args, shape):
                        "attn_impl": "auto"},
             "clocks": clocks,
             "e2e": {"value": total_bytes / (e2e_ms * 1e-3) / 1e9 if e2e_ms else None, "unit": "GB/s", "ms_per_step": e2e_ms,
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "call": "tts_verify_step_host, fp32 probabilities"},
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "call": "tts_verify_step_host, fp32 probabilities in pinned host memory: copied are the queries and the small "
+                            "arrays; of the %d bytes of probabilities the accept kernel reads its %d algorithmic bytes in place"
+                            % ((h_p.numel() + h_q.numel()) * 4 if ds.with_accept else 0, acc_bytes)},
             "e2e_logits": e2e_logits,
             "gpu_launches": launches,
             "roofline": roof,

@@ -377,7 +377,9 @@ TTS_API int tts_kv_rollback(tts_ctx* ctx, int32_t* branch_lens, const int32_t* a
  * streams of its own on which the copies that need not wait for the kernels run beside them (the
  * queries of later layers and the accept inputs while the first layers run, the outputs of finished
  * layers while later ones run); the kernels run on the context's stream.  With pageable host memory
- * the copies do not overlap anything.
+ * the copies do not overlap anything.  When p_target_host and q_draft_host are pinned memory that the
+ * device can address (cudaHostAlloc / cudaHostRegister), they are not copied at all: the accept kernel
+ * reads what it needs of them (its 2 gamma gathers and one row pair per branch) directly from the host.
  */
 TTS_API int tts_verify_step_host(tts_ctx* ctx, int n_layers, const void* q_host, const void* const* k_pools,
                          const void* const* v_pools, const int32_t* block_table_host,

@@ -757,9 +757,24 @@ int step_host(tts_ctx* ctx, int n_layers, const void* q_host, const void* const*
         TTS_CK(copy_q(l0, l1, up_st));
         TTS_CK(cudaEventRecord(ev_q[ch], up_st));
     }
-    TTS_CK(cudaMemcpyAsync(d_pt, p_target_host, (size_t)n_branches * (gamma + 1) * vocab * dist_elt, cudaMemcpyHostToDevice, up_st));
+    // Probabilities in pinned (device-mapped) host memory are not copied: the accept kernel reads, straight from the
+    // host, the 2 gamma scalars of its tests and the one row pair of its draw, a quarter of the two tensors, instead
+    // of all of them crossing the link behind the queries.  (The logits variant reads its rows twice: it copies.)
+    const void* p_dev = nullptr; const void* q_dev = nullptr;
+    bool zero_copy = false;
+    if (logits_dtype < 0) {
+        void* a = nullptr; void* b = nullptr;
+        zero_copy = cudaHostGetDevicePointer(&a, const_cast<void*>(p_target_host), 0) == cudaSuccess &&
+                    (gamma == 0 || cudaHostGetDevicePointer(&b, const_cast<void*>(q_draft_host), 0) == cudaSuccess);
+        if (!zero_copy) (void)cudaGetLastError();            // pageable memory: not an error of this call
+        zero_copy = zero_copy && aligned16(a) && (gamma == 0 || aligned16(b));
+        p_dev = a; q_dev = b;
+    }
+    if (!zero_copy)
+        TTS_CK(cudaMemcpyAsync(d_pt, p_target_host, (size_t)n_branches * (gamma + 1) * vocab * dist_elt, cudaMemcpyHostToDevice, up_st));
     if (gamma > 0) {
-        TTS_CK(cudaMemcpyAsync(d_qd, q_draft_host, (size_t)n_branches * gamma * vocab * dist_elt, cudaMemcpyHostToDevice, up_st));
+        if (!zero_copy)
+            TTS_CK(cudaMemcpyAsync(d_qd, q_draft_host, (size_t)n_branches * gamma * vocab * dist_elt, cudaMemcpyHostToDevice, up_st));
         TTS_CK(cudaMemcpyAsync(d_dt, draft_tokens_host, (size_t)n_branches * gamma * 4, cudaMemcpyHostToDevice, up_st));
     }
     TTS_CK(cudaMemcpyAsync(d_un, uniforms_host, (size_t)n_branches * (gamma + 1) * 4, cudaMemcpyHostToDevice, up_st));
@@ -784,7 +799,8 @@ int step_host(tts_ctx* ctx, int n_layers, const void* q_host, const void* const*
     }
     TTS_CK(cudaStreamWaitEvent(st, ev_acc, 0));
     int rc = logits_dtype < 0
-                 ? tts_accept(ctx, (const float*)d_pt, gamma > 0 ? (const float*)d_qd : nullptr, gamma > 0 ? d_dt : nullptr, d_un,
+                 ? tts_accept(ctx, zero_copy ? (const float*)p_dev : (const float*)d_pt,
+                              gamma > 0 ? (zero_copy ? (const float*)q_dev : (const float*)d_qd) : nullptr, gamma > 0 ? d_dt : nullptr, d_un,
                               n_branches, gamma, vocab, d_al, d_nt)
                  : tts_accept_logits(ctx, d_pt, gamma > 0 ? d_qd : nullptr, logits_dtype, gamma > 0 ? d_dt : nullptr, d_un,
                                      n_branches, gamma, vocab, d_al, d_nt);
